@@ -1,0 +1,161 @@
+/* libbuzz -- C ABI of the BUZZ sparse KV-cache hot path on one NVIDIA B200 (sm_100a).
+ *
+ * BUZZ (arXiv 2410.23079) keeps, per attention head, a bounded KV cache laid out in position
+ * order as  [ sink | old | new | window ]  (Algorithm 1): the first `sink` tokens, survivors of
+ * earlier evictions ("old"), tokens that left the sliding window since the last eviction ("new"),
+ * and the last `window` tokens. Each retained token carries an accumulated attention score
+ * (Algorithm 2's input A). When the cache is full, the new tokens are cut into segments of
+ * `segment` tokens and the top-scoring `hitters` of each segment survive, while the old tokens are
+ * thinned to every s_hat-th, s_hat = floor((segment+1)/2) (Section 3.3).
+ *
+ * Conventions for every call:
+ *   - All tensor pointers are DEVICE pointers unless the name says `_host`. The caller allocates
+ *     and owns all device memory and the stream; the library allocates no device memory, creates
+ *     no stream, and (except where stated) does not synchronise.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *   - Return value: BUZZ_OK or a negative BUZZ_ERR_* code. Nothing throws, traps or aborts.
+ *     Conditions found on the device (slot overflow, an eviction that cannot shrink the cache)
+ *     are recorded in a device status word, the affected sequence is left untouched, and the
+ *     code surfaces at buzz_status().
+ *   - Element type `dtype`: BUZZ_F32 (4-byte IEEE) or BUZZ_BF16 (2-byte bfloat16) for Q/K/V/O and
+ *     the caches; scores are always fp32, positions int32. All pointers must be 16-byte aligned.
+ *   - One instance = (layer, sequence, KV head). With grouped-query attention the q_heads/kv_heads
+ *     query heads of a group share the instance and their probabilities are summed into one score.
+ */
+#ifndef BUZZ_H_
+#define BUZZ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum { BUZZ_F32 = 0, BUZZ_BF16 = 1 };
+
+enum {
+  BUZZ_OK = 0,
+  BUZZ_ERR_INVALID = -1,     /* bad argument (synchronous, nothing was launched)            */
+  BUZZ_ERR_OVERFLOW = -2,    /* decode step on a full cache (evict was not called in time)   */
+  BUZZ_ERR_NO_PROGRESS = -3, /* an eviction left the cache full (degenerate parameters)      */
+  BUZZ_ERR_TIMEOUT = -4,     /* a bounded on-device wait expired                             */
+  BUZZ_ERR_CUDA = -5         /* a CUDA runtime call failed                                   */
+};
+
+typedef struct buzz_ctx* buzz_t;
+
+typedef struct buzz_shape {
+  int32_t layers;            /* L                                                            */
+  int32_t max_batch;         /* sequences per layer the caches are sized for                 */
+  int32_t q_heads;           /* Hq                                                           */
+  int32_t kv_heads;          /* Hkv, must divide Hq                                          */
+  int32_t head_dim;          /* d: 64 or 128                                                 */
+  int32_t dtype;             /* BUZZ_F32 or BUZZ_BF16                                        */
+  int32_t max_prompt_tokens; /* upper bound on the packed token count of one buzz_prefill    */
+  int32_t flags;             /* BUZZ_FLAG_*                                                  */
+} buzz_shape;
+
+enum {
+  BUZZ_FLAG_LOGN = 1         /* scale logits by log_512(tokens seen)/sqrt(d) (Section 3.5)   */
+};
+
+/* Sizes of the two device allocations buzz_create needs (Section 3.3 fixes the cache at
+ * budget = T + sink + window slots per instance).
+ *   state   : K and V caches [L][max_batch][Hkv][budget][d], score and pos [L][max_batch][Hkv][budget],
+ *             counters n / n_old / total_len [L][max_batch][Hkv], and the status words.
+ *   scratch : per-row softmax statistics and per-key column sums of one prefill, plus staging
+ *             buffers for buzz_decode_step_host. Contents are not carried between calls.
+ * Returns BUZZ_ERR_INVALID for a shape or budget the library does not support. */
+int buzz_workspace_bytes(const buzz_shape* shape, int budget, size_t* state_bytes, size_t* scratch_bytes);
+
+/* Creates a cache policy object (Table 1: k = sink, w = window, s = segment; budget = T + k + w,
+ * Remark 2). `hitters` is the number of winners kept per segment. Both allocations must be at
+ * least as large as buzz_workspace_bytes reports and 256-byte aligned; `state_dev` is zeroed here
+ * (one synchronous memset on the default stream). Rejects: sink < 0, window < 1, segment < 2,
+ * hitters < 1, hitters >= segment, budget < sink + window + segment, kv_heads not dividing
+ * q_heads, head_dim not in {64, 128}, undersized or misaligned buffers. */
+int buzz_create(buzz_t* out, int sink, int window, int segment, int hitters, int budget,
+                const buzz_shape* shape, void* state_dev, size_t state_bytes,
+                void* scratch_dev, size_t scratch_bytes);
+
+/* Frees the host object only. */
+void buzz_destroy(buzz_t ctx);
+
+/* Prefill of one layer (Eqs. 1 and 3; Remark 2).
+ *   q  [total_tokens][Hq][d], k, v [total_tokens][Hkv][d], out [total_tokens][Hq][d], all packed
+ *   over `batch` sequences by cu_seqlens_dev [batch+1] (int32, device; cu[0] = 0).
+ * Computes causal attention out = Softmax(q k^T / sqrt(d)) v per sequence and head, the initial
+ * score of every key = the sum of the probabilities it received (column sums, summed over the
+ * query heads of its group, in a fixed order), then, while a sequence holds >= budget tokens,
+ * eviction rounds (first round: segment-wise top-`hitters` over everything between sink and
+ * window; later rounds: every s_hat-th survivor), and writes the survivors' K, V, score and
+ * position into the layer's cache. Resets that layer's sequences 0..batch-1.
+ * `max_seqlen` is an upper bound on any sequence's length (host value, used for grid sizing). */
+int buzz_prefill(buzz_t ctx, int layer, const void* q, const void* k, const void* v,
+                 const int32_t* cu_seqlens_dev, int batch, int total_tokens, int max_seqlen,
+                 void* out, void* stream);
+
+/* One decode step of one layer (Eqs. 2 and 3) for the `batch` sequences of the last prefill:
+ *   q [batch][Hq][d], k_new, v_new [batch][Hkv][d], out [batch][Hq][d].
+ * Appends (k_new, v_new) at slot n with score 0 and position total_len, attends over all n+1
+ * retained slots, and adds each slot's probability (summed over the group's query heads) to its
+ * score. A sequence whose cache is already full is skipped and BUZZ_ERR_OVERFLOW is recorded. */
+int buzz_decode_step(buzz_t ctx, int layer, const void* q, const void* k_new, const void* v_new,
+                     void* out, void* stream);
+
+/* The same step with HOST buffers (pinned memory recommended): copies q/k_new/v_new to the
+ * library's staging area in scratch, runs the step, copies `out` back, all on `stream`, without
+ * synchronising. Layouts as in buzz_decode_step. */
+int buzz_decode_step_host(buzz_t ctx, int layer, const void* q_host, const void* k_new_host,
+                          const void* v_new_host, void* out_host, void* stream);
+
+/* BUZZ eviction (Algorithm 1's sampling line and final concatenation; Algorithm 2) for one layer,
+ * or for all layers when layer = -1. Per instance, entirely on the device: nothing happens unless
+ * n >= budget (threshold buffering, Section 3.3) and n > sink + window (Remark 1). Otherwise the
+ * old region keeps offsets 0, s_hat, 2 s_hat, ...; the new region [sink + n_old, n - window) is
+ * cut into segments of `segment` slots (a short last one allowed) and each keeps its top
+ * min(hitters, length) slots by (score descending, position ascending), emitted in position order;
+ * K, V, score and pos are compacted in place as sink | old' | new' | window; n_old becomes
+ * |old'| + |new'|. Calling it after every decode step is the intended use. */
+int buzz_evict(buzz_t ctx, int layer, void* stream);
+
+/* Test/checkpoint getter for one instance. Synchronises `stream`-independent: it waits for the
+ * device. Any output pointer may be NULL. pos_host/score_host receive n entries, k_host/v_host
+ * n*d elements of the cache dtype, in slot order (= position order). Buffers must hold `budget`
+ * entries. */
+int buzz_export_state(buzz_t ctx, int layer, int seq, int kv_head, int32_t* n, int32_t* n_old,
+                      int32_t* total_len, int32_t* pos_host, float* score_host, void* k_host,
+                      void* v_host);
+
+/* The inverse of buzz_export_state (checkpoint restore, and how tests plant a cache state): loads
+ * n slots (n <= budget, n_old <= n, total_len >= n) of one instance from host buffers laid out as
+ * buzz_export_state writes them, and marks sequences 0..seq of the layer active. Waits for the
+ * device before and after copying. */
+int buzz_import_state(buzz_t ctx, int layer, int seq, int kv_head, int32_t n, int32_t n_old,
+                      int32_t total_len, const int32_t* pos_host, const float* score_host,
+                      const void* k_host, const void* v_host);
+
+/* Copies the pre-eviction prompt scores of the last buzz_prefill (one fp32 per prompt token of
+ * KV head `kv_head`, packed like the prompt) to score_host [total_tokens]. Waits for the device. */
+int buzz_export_prefill_scores(buzz_t ctx, int kv_head, int total_tokens, float* score_host);
+
+/* Waits for `stream`, then returns the first error recorded on the device since the last call
+ * (BUZZ_OK if none) and clears it. */
+int buzz_status(buzz_t ctx, void* stream);
+
+/* Number of kernels the library has launched through this object (for launch accounting). */
+int64_t buzz_launch_count(buzz_t ctx);
+
+/* Tuning knob: number of CTAs (1, 2, 4 or 8) of the thread-block cluster that shares one instance's
+ * slots in buzz_decode_step; 0 restores the built-in choice. Results do not depend on it beyond
+ * fp32 summation order. */
+int buzz_set_decode_cluster(buzz_t ctx, int cluster_size);
+
+/* Static description of an error code. */
+const char* buzz_error_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BUZZ_H_ */

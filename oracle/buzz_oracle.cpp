@@ -235,7 +235,7 @@ void bo_set_scores(void* p, const double* score) {
 int bo_set_state(void* p, int n, int n_old, int total_len, const int32_t* pos, const double* score,
                  const double* K, const double* V) {
   Head& h = *(Head*)p;
-  if (n < 0 || n > h.budget || n_old < 0) return BO_BAD_ARG;
+  if (n < 0 || n_old < 0 || n_old > n) return BO_BAD_ARG;   // n may exceed the budget (a prompt)
   h.n = n; h.n_old = n_old; h.total_len = total_len;
   h.pos.assign(pos, pos + n);
   h.score.assign(score, score + n);

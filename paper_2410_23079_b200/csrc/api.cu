@@ -1,0 +1,279 @@
+// libbuzz C ABI: argument checking, workspace partitioning and kernel dispatch.
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "buzz_internal.cuh"
+
+cudaError_t buzz_launch_prefill_simt(buzz_ctx* c, const void* q, const void* k, const void* v,
+                                     const int32_t* cu, int batch, int max_seqlen, void* out,
+                                     cudaStream_t stream, int* launches);
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Layout {
+  size_t k, v, score, pos, n, n_old, total, status, state_bytes;
+  size_t lse, pscore, stage, scratch_bytes, stage_q, stage_kv;
+};
+
+bool shape_ok(const buzz_shape* s, int budget) {
+  if (!s) return false;
+  if (s->layers < 1 || s->max_batch < 1 || s->q_heads < 1 || s->kv_heads < 1) return false;
+  if (s->q_heads % s->kv_heads) return false;
+  const int g = s->q_heads / s->kv_heads;
+  if (g != 1 && g != 2 && g != 4 && g != 8) return false;
+  if (s->head_dim != 64 && s->head_dim != 128) return false;
+  if (s->dtype != BUZZ_F32 && s->dtype != BUZZ_BF16) return false;
+  if (s->max_prompt_tokens < 1) return false;
+  if (budget < 1 || budget > 32768) return false;
+  return true;
+}
+
+Layout make_layout(const buzz_shape& s, int budget) {
+  Layout L{};
+  const size_t e = s.dtype == BUZZ_BF16 ? 2 : 4;
+  const size_t inst = (size_t)s.layers * s.max_batch * s.kv_heads;
+  size_t off = 0;
+  L.k = off; off = align_up(off + inst * budget * s.head_dim * e);
+  L.v = off; off = align_up(off + inst * budget * s.head_dim * e);
+  L.score = off; off = align_up(off + inst * budget * sizeof(float));
+  L.pos = off; off = align_up(off + inst * budget * sizeof(int32_t));
+  L.n = off; off = align_up(off + inst * sizeof(int32_t));
+  L.n_old = off; off = align_up(off + inst * sizeof(int32_t));
+  L.total = off; off = align_up(off + inst * sizeof(int32_t));
+  L.status = off; off = align_up(off + 4 * sizeof(int32_t));
+  L.state_bytes = off;
+  off = 0;
+  L.lse = off; off = align_up(off + (size_t)s.q_heads * s.max_prompt_tokens * sizeof(float));
+  L.pscore = off; off = align_up(off + (size_t)s.kv_heads * s.max_prompt_tokens * sizeof(float));
+  L.stage_q = align_up((size_t)s.max_batch * s.q_heads * s.head_dim * e);
+  L.stage_kv = align_up((size_t)s.max_batch * s.kv_heads * s.head_dim * e);
+  L.stage = off; off += 2 * L.stage_q + 2 * L.stage_kv;
+  L.scratch_bytes = off;
+  return L;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+int buzz_workspace_bytes(const buzz_shape* shape, int budget, size_t* state_bytes, size_t* scratch_bytes) {
+  if (!shape_ok(shape, budget) || !state_bytes || !scratch_bytes) return BUZZ_ERR_INVALID;
+  const Layout L = make_layout(*shape, budget);
+  *state_bytes = L.state_bytes;
+  *scratch_bytes = L.scratch_bytes;
+  return BUZZ_OK;
+}
+
+int buzz_create(buzz_t* out, int sink, int window, int segment, int hitters, int budget,
+                const buzz_shape* shape, void* state_dev, size_t state_bytes, void* scratch_dev,
+                size_t scratch_bytes) {
+  if (!out) return BUZZ_ERR_INVALID;
+  *out = nullptr;
+  if (!shape_ok(shape, budget)) return BUZZ_ERR_INVALID;
+  if (sink < 0 || window < 1 || segment < 2 || segment > 1024 || hitters < 1 || hitters >= segment)
+    return BUZZ_ERR_INVALID;
+  if (budget < sink + window + segment) return BUZZ_ERR_INVALID;
+  const Layout L = make_layout(*shape, budget);
+  if (!state_dev || !scratch_dev || state_bytes < L.state_bytes || scratch_bytes < L.scratch_bytes)
+    return BUZZ_ERR_INVALID;
+  if ((reinterpret_cast<uintptr_t>(state_dev) | reinterpret_cast<uintptr_t>(scratch_dev)) & (kAlign - 1))
+    return BUZZ_ERR_INVALID;
+  buzz_ctx* c = new (std::nothrow) buzz_ctx();
+  if (!c) return BUZZ_ERR_INVALID;
+  c->pol = BuzzPolicy{sink, window, segment, hitters, budget, (segment + 1) / 2};
+  c->sh = *shape;
+  c->group = shape->q_heads / shape->kv_heads;
+  c->esize = shape->dtype == BUZZ_BF16 ? 2 : 4;
+  char* sb = static_cast<char*>(state_dev);
+  c->st.K = sb + L.k;
+  c->st.V = sb + L.v;
+  c->st.score = reinterpret_cast<float*>(sb + L.score);
+  c->st.pos = reinterpret_cast<int32_t*>(sb + L.pos);
+  c->st.n = reinterpret_cast<int32_t*>(sb + L.n);
+  c->st.n_old = reinterpret_cast<int32_t*>(sb + L.n_old);
+  c->st.total = reinterpret_cast<int32_t*>(sb + L.total);
+  c->st.status = reinterpret_cast<int32_t*>(sb + L.status);
+  char* sc = static_cast<char*>(scratch_dev);
+  c->lse = reinterpret_cast<float*>(sc + L.lse);
+  c->pscore = reinterpret_cast<float*>(sc + L.pscore);
+  c->stage = sc + L.stage;
+  c->stage_q = L.stage_q;
+  c->stage_kv = L.stage_kv;
+  c->batch = static_cast<int*>(calloc(shape->layers, sizeof(int)));
+  c->decode_cluster = 0;
+  c->launches = 0;
+  if (!c->batch) { delete c; return BUZZ_ERR_INVALID; }
+  if (cudaMemset(state_dev, 0, L.state_bytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+    free(c->batch);
+    delete c;
+    return BUZZ_ERR_CUDA;
+  }
+  *out = c;
+  return BUZZ_OK;
+}
+
+void buzz_destroy(buzz_t c) {
+  if (!c) return;
+  free(c->batch);
+  delete c;
+}
+
+int buzz_prefill(buzz_t c, int layer, const void* q, const void* k, const void* v,
+                 const int32_t* cu_seqlens_dev, int batch, int total_tokens, int max_seqlen,
+                 void* out, void* stream) {
+  if (!c || layer < 0 || layer >= c->sh.layers || batch < 1 || batch > c->sh.max_batch) return BUZZ_ERR_INVALID;
+  if (total_tokens < 1 || total_tokens > c->sh.max_prompt_tokens || max_seqlen < 1 || max_seqlen > total_tokens)
+    return BUZZ_ERR_INVALID;
+  if (!q || !k || !v || !out || !cu_seqlens_dev) return BUZZ_ERR_INVALID;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return BUZZ_ERR_INVALID;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int launches = 0;
+  cudaError_t e;
+  e = buzz_launch_prefill_simt(c, q, k, v, cu_seqlens_dev, batch, max_seqlen, out, s, &launches);
+  c->launches += launches;
+  if (e != cudaSuccess) return BUZZ_ERR_CUDA;
+  c->batch[layer] = batch;
+  e = buzz_launch_prefill_fill(c, layer, k, v, cu_seqlens_dev, batch, max_seqlen, s);
+  return e == cudaSuccess ? BUZZ_OK : BUZZ_ERR_CUDA;
+}
+
+int buzz_decode_step(buzz_t c, int layer, const void* q, const void* k_new, const void* v_new,
+                     void* out, void* stream) {
+  if (!c || layer < 0 || layer >= c->sh.layers || !q || !k_new || !v_new || !out) return BUZZ_ERR_INVALID;
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return BUZZ_ERR_INVALID;
+  cudaError_t e = buzz_launch_decode(c, layer, q, k_new, v_new, out, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? BUZZ_OK : BUZZ_ERR_CUDA;
+}
+
+int buzz_decode_step_host(buzz_t c, int layer, const void* q_host, const void* k_new_host,
+                          const void* v_new_host, void* out_host, void* stream) {
+  if (!c || layer < 0 || layer >= c->sh.layers || !q_host || !k_new_host || !v_new_host || !out_host)
+    return BUZZ_ERR_INVALID;
+  const int batch = c->batch[layer];
+  if (batch == 0) return BUZZ_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t qb = (size_t)batch * c->sh.q_heads * c->sh.head_dim * c->esize;
+  const size_t kb = (size_t)batch * c->sh.kv_heads * c->sh.head_dim * c->esize;
+  char* dq = c->stage;
+  char* dk = dq + c->stage_q;
+  char* dv = dk + c->stage_kv;
+  char* dout = dv + c->stage_kv;
+  if (cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (buzz_launch_decode(c, layer, dq, dk, dv, dout, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+  return BUZZ_OK;
+}
+
+int buzz_evict(buzz_t c, int layer, void* stream) {
+  if (!c || layer < -1 || layer >= c->sh.layers) return BUZZ_ERR_INVALID;
+  cudaError_t e = layer < 0 ? buzz_launch_evict(c, 0, c->sh.layers, static_cast<cudaStream_t>(stream))
+                            : buzz_launch_evict(c, layer, 1, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? BUZZ_OK : BUZZ_ERR_CUDA;
+}
+
+int buzz_export_state(buzz_t c, int layer, int seq, int kv_head, int32_t* n, int32_t* n_old,
+                      int32_t* total_len, int32_t* pos_host, float* score_host, void* k_host,
+                      void* v_host) {
+  if (!c || layer < 0 || layer >= c->sh.layers || seq < 0 || seq >= c->sh.max_batch || kv_head < 0 ||
+      kv_head >= c->sh.kv_heads)
+    return BUZZ_ERR_INVALID;
+  if (cudaDeviceSynchronize() != cudaSuccess) return BUZZ_ERR_CUDA;
+  const size_t inst = buzz_inst(c->sh, layer, seq, kv_head);
+  int32_t cnt[3];
+  if (cudaMemcpy(&cnt[0], c->st.n + inst, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (cudaMemcpy(&cnt[1], c->st.n_old + inst, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (cudaMemcpy(&cnt[2], c->st.total + inst, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (n) *n = cnt[0];
+  if (n_old) *n_old = cnt[1];
+  if (total_len) *total_len = cnt[2];
+  const int m = cnt[0];
+  if (m < 0 || m > c->pol.budget) return BUZZ_ERR_INVALID;
+  const size_t row = (size_t)c->sh.head_dim * c->esize;
+  const size_t slot0 = inst * c->pol.budget;
+  if (m > 0) {
+    if (pos_host && cudaMemcpy(pos_host, c->st.pos + slot0, (size_t)m * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (score_host && cudaMemcpy(score_host, c->st.score + slot0, (size_t)m * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (k_host && cudaMemcpy(k_host, c->st.K + slot0 * row, m * row, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (v_host && cudaMemcpy(v_host, c->st.V + slot0 * row, m * row, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
+  }
+  return BUZZ_OK;
+}
+
+int buzz_import_state(buzz_t c, int layer, int seq, int kv_head, int32_t n, int32_t n_old,
+                      int32_t total_len, const int32_t* pos_host, const float* score_host,
+                      const void* k_host, const void* v_host) {
+  if (!c || layer < 0 || layer >= c->sh.layers || seq < 0 || seq >= c->sh.max_batch || kv_head < 0 ||
+      kv_head >= c->sh.kv_heads)
+    return BUZZ_ERR_INVALID;
+  if (n < 0 || n > c->pol.budget || n_old < 0 || n_old > n || total_len < n) return BUZZ_ERR_INVALID;
+  if (n > 0 && (!pos_host || !score_host || !k_host || !v_host)) return BUZZ_ERR_INVALID;
+  if (cudaDeviceSynchronize() != cudaSuccess) return BUZZ_ERR_CUDA;
+  const size_t inst = buzz_inst(c->sh, layer, seq, kv_head);
+  const size_t row = (size_t)c->sh.head_dim * c->esize;
+  const size_t slot0 = inst * c->pol.budget;
+  if (n > 0) {
+    if (cudaMemcpy(c->st.pos + slot0, pos_host, (size_t)n * 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (cudaMemcpy(c->st.score + slot0, score_host, (size_t)n * 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (cudaMemcpy(c->st.K + slot0 * row, k_host, n * row, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (cudaMemcpy(c->st.V + slot0 * row, v_host, n * row, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
+  }
+  const int32_t cnt[3] = {n, n_old, total_len};
+  if (cudaMemcpy(c->st.n + inst, &cnt[0], 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (cudaMemcpy(c->st.n_old + inst, &cnt[1], 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (cudaMemcpy(c->st.total + inst, &cnt[2], 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (c->batch[layer] < seq + 1) c->batch[layer] = seq + 1;
+  return BUZZ_OK;
+}
+
+int buzz_export_prefill_scores(buzz_t c, int kv_head, int total_tokens, float* score_host) {
+  if (!c || kv_head < 0 || kv_head >= c->sh.kv_heads || total_tokens < 1 ||
+      total_tokens > c->sh.max_prompt_tokens || !score_host)
+    return BUZZ_ERR_INVALID;
+  if (cudaDeviceSynchronize() != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (cudaMemcpy(score_host, c->pscore + (size_t)kv_head * c->sh.max_prompt_tokens,
+                 (size_t)total_tokens * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return BUZZ_ERR_CUDA;
+  return BUZZ_OK;
+}
+
+int buzz_status(buzz_t c, void* stream) {
+  if (!c) return BUZZ_ERR_INVALID;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return BUZZ_ERR_CUDA;
+  int32_t word[4];
+  if (cudaMemcpy(word, c->st.status, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (word[0] != 0 && cudaMemset(c->st.status, 0, sizeof(word)) != cudaSuccess) return BUZZ_ERR_CUDA;
+  return word[0];
+}
+
+int64_t buzz_launch_count(buzz_t c) { return c ? c->launches : 0; }
+
+int buzz_set_decode_cluster(buzz_t c, int cluster_size) {
+  if (!c) return BUZZ_ERR_INVALID;
+  if (cluster_size != 0 && cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8)
+    return BUZZ_ERR_INVALID;
+  c->decode_cluster = cluster_size;
+  return BUZZ_OK;
+}
+
+const char* buzz_error_string(int code) {
+  switch (code) {
+    case BUZZ_OK: return "ok";
+    case BUZZ_ERR_INVALID: return "invalid argument";
+    case BUZZ_ERR_OVERFLOW: return "decode step on a full cache (call buzz_evict after every step)";
+    case BUZZ_ERR_NO_PROGRESS: return "eviction cannot shrink the cache (segment too small for this budget)";
+    case BUZZ_ERR_TIMEOUT: return "a bounded on-device wait expired";
+    case BUZZ_ERR_CUDA: return "a CUDA runtime call failed";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

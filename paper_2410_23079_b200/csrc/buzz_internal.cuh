@@ -1,0 +1,71 @@
+// Internal definitions shared by the libbuzz translation units (host object, device views,
+// launch wrappers). Not part of the public ABI.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "buzz.h"
+
+// BUZZ policy constants as the kernels see them (Table 1 of the paper).
+struct BuzzPolicy {
+  int sink;      // k
+  int window;    // w
+  int segment;   // s
+  int hitters;   // winners per segment
+  int budget;    // T + k + w
+  int s_hat;     // floor((s+1)/2)
+};
+
+// Device view of the persistent state. Instance index = ((layer * max_batch) + seq) * kv_heads + head.
+struct BuzzState {
+  char* K;            // [inst][budget][d] elements
+  char* V;            // [inst][budget][d] elements
+  float* score;       // [inst][budget]
+  int32_t* pos;       // [inst][budget]
+  int32_t* n;         // [inst] retained slots
+  int32_t* n_old;     // [inst] slots between sink and window that survived an eviction
+  int32_t* total;     // [inst] tokens seen so far (next position)
+  int32_t* status;    // [4]: first error code, instance, detail, spare
+};
+
+struct buzz_ctx {
+  BuzzPolicy pol;
+  buzz_shape sh;
+  int group;          // q_heads / kv_heads
+  size_t esize;       // bytes per K/V element
+  BuzzState st;
+  // scratch partition
+  float* lse;         // [q_heads][max_prompt_tokens] row log-sum-exp (log2 domain) of one prefill
+  float* pscore;      // [kv_heads][max_prompt_tokens] pre-eviction prompt scores
+  char* stage;        // staging for buzz_decode_step_host: q | k | v | out
+  size_t stage_q, stage_kv;  // byte sizes of one q-shaped and one kv-shaped staging tensor
+  int* batch;         // active sequences per layer (host array)
+  int decode_cluster; // 0 = choose automatically
+  long long launches;
+};
+
+__host__ __device__ inline size_t buzz_inst(const buzz_shape& sh, int layer, int seq, int head) {
+  return ((size_t)layer * sh.max_batch + seq) * sh.kv_heads + head;
+}
+
+// Records the first error seen on the device; later ones are dropped.
+__device__ inline void buzz_set_status(int32_t* status, int code, int inst, int detail) {
+  if (atomicCAS(status, 0, code) == 0) {
+    status[1] = inst;
+    status[2] = detail;
+  }
+}
+
+// ---- launch wrappers (each returns a cudaError_t from the launch) ---------------------------
+cudaError_t buzz_launch_decode(buzz_ctx* c, int layer, const void* q, const void* k_new,
+                               const void* v_new, void* out, cudaStream_t stream);
+cudaError_t buzz_launch_evict(buzz_ctx* c, int layer_begin, int layer_count, cudaStream_t stream);
+cudaError_t buzz_launch_prefill_attention(buzz_ctx* c, const void* q, const void* k, const void* v,
+                                          const int32_t* cu, int batch, int total_tokens,
+                                          int max_seqlen, void* out, cudaStream_t stream,
+                                          int* launches);
+cudaError_t buzz_launch_prefill_fill(buzz_ctx* c, int layer, const void* k, const void* v,
+                                     const int32_t* cu, int batch, int max_seqlen,
+                                     cudaStream_t stream);

@@ -1,0 +1,143 @@
+"""Lock-step comparison of libbuzz (CUDA) against the CPU oracle on one workload.
+
+Both sides receive the same seeded inputs (the GPU tensors' bytes, copied to the host). For every
+sampled (layer, sequence, KV head) instance:
+  * prefill outputs and pre-eviction prompt scores are compared within tolerance;
+  * selection parity is lock-step: the GPU's fp32 scores are loaded into a second oracle instance,
+    which then takes every arg-max decision on exactly the values the GPU holds; retained
+    positions, counters, scores and K/V rows must then match bit for bit;
+  * every decode step's output is compared within tolerance, the running scores to rel 1e-3, and
+    before each eviction the oracle's scores are replaced by the GPU's (lock-step again).
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import workloads
+from oracle.buzz_oracle import OracleHead
+from paper_2410_23079_b200 import Buzz
+
+TOL = {"bf16": dict(atol=2e-2, rtol=1e-2), "f32": dict(atol=1e-4, rtol=1e-4)}
+SCORE_RTOL = 1e-3
+
+
+def make_buzz(w: workloads.Workload, device="cuda:0", max_prompt_tokens=None, logn=False) -> Buzz:
+    dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    lens = workloads.prompt_lengths(w)
+    return Buzz(sink=w.sink, window=w.window, segment=w.segment, hitters=w.hitters, budget=w.budget,
+                layers=w.layers, max_batch=w.batch, q_heads=w.q_heads, kv_heads=w.kv_heads,
+                head_dim=w.head_dim, dtype=dt, max_prompt_tokens=max_prompt_tokens or sum(lens),
+                logn=logn, device=device)
+
+
+def _np64(t: torch.Tensor) -> np.ndarray:
+    return t.detach().to("cpu", torch.float64).numpy()
+
+
+def assert_close(got, ref, atol, rtol, what):
+    got, ref = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
+    err = np.abs(got - ref)
+    bad = err > atol + rtol * np.abs(ref)
+    assert not bad.any(), f"{what}: {bad.sum()} of {bad.size} off, max abs err {err.max():.3e}"
+
+
+def assert_scores_close(got, ref, what):
+    got, ref = np.asarray(got, dtype=np.float64), np.asarray(ref, dtype=np.float64)
+    rel = np.abs(got - ref) / np.maximum(np.abs(ref), 1e-30)
+    assert rel.max(initial=0.0) <= SCORE_RTOL, f"{what}: max rel err {rel.max():.3e}"
+
+
+def compare_state(bz: Buzz, orc: OracleHead, layer, seq, head, what, exact_scores):
+    st = bz.export_state(layer, seq, head)
+    n, n_old, tot = orc.counts()
+    assert (st["n"], st["n_old"], st["total_len"]) == (n, n_old, tot), f"{what}: counters {st['n'], st['n_old'], st['total_len']} vs {(n, n_old, tot)}"
+    pos, score, K, V = orc.state()
+    assert np.array_equal(st["pos"].numpy(), pos), f"{what}: retained positions differ"
+    assert np.array_equal(_np64(st["k"]), K) and np.array_equal(_np64(st["v"]), V), f"{what}: K/V rows differ"
+    if exact_scores:
+        assert np.array_equal(st["score"].numpy().astype(np.float64), score), f"{what}: scores differ"
+    else:
+        assert_scores_close(st["score"].numpy(), score, what + " scores")
+    return st
+
+
+def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None, check_every=1,
+                 device="cuda:0", logn=False, bz: Buzz | None = None):
+    """Runs prefill + decode/evict on the GPU for the whole workload and the oracle on `samples`
+    (a list of (layer, seq, kv_head)). Returns a dict of summary counters."""
+    tol = TOL[w.dtype]
+    S = w.decode_steps if decode_steps is None else decode_steps
+    layers = list(range(w.layers)) if layers is None else layers
+    own = bz is None
+    bz = bz or make_buzz(w, device, logn=logn)
+    lens = workloads.prompt_lengths(w)
+    offs = np.concatenate([[0], np.cumsum(lens)])
+    g, d = w.group, w.head_dim
+    stats = dict(evictions=0, prefill_rounds=0, max_out_err=0.0)
+    lock = {}
+    dec = {}
+    for layer in layers:
+        q, k, v, cu = workloads.prefill_inputs(w, layer, device)
+        out = torch.empty_like(q)
+        bz.prefill(layer, q, k, v, cu, max(lens), out)
+        assert bz.status() == 0
+        dec[layer] = workloads.decode_inputs(w, layer, device, steps=S)
+        pscore = {}
+        for (ll, b, h) in samples:
+            if ll != layer:
+                continue
+            a, e = int(offs[b]), int(offs[b + 1])
+            Q = _np64(q[a:e, h * g:(h + 1) * g]).transpose(1, 0, 2)
+            K, V = _np64(k[a:e, h]), _np64(v[a:e, h])
+            free = OracleHead(g, d, w.sink, w.window, w.segment, w.hitters, w.budget, logn=logn)
+            O, full, rounds = free.prefill(Q, K, V)
+            stats["prefill_rounds"] = max(stats["prefill_rounds"], rounds)
+            got = _np64(out[a:e, h * g:(h + 1) * g]).transpose(1, 0, 2)
+            assert_close(got, O, what=f"prefill out L{layer} b{b} h{h}", **tol)
+            stats["max_out_err"] = max(stats["max_out_err"], float(np.abs(got - O).max()))
+            if h not in pscore:
+                pscore[h] = bz.export_prefill_scores(h, int(offs[-1])).numpy()
+            gs = pscore[h][a:e]
+            assert_scores_close(gs, full, f"prefill scores L{layer} b{b} h{h}")
+            # lock-step instance: selection decided on the GPU's fp32 scores
+            ls = OracleHead(g, d, w.sink, w.window, w.segment, w.hitters, w.budget, logn=logn)
+            N = e - a
+            ls.set_state(0, N, np.arange(N), gs.astype(np.float64), K, V)
+            while ls.counts()[0] >= w.budget:
+                assert ls.evict() == 1
+            compare_state(bz, ls, layer, b, h, f"after prefill L{layer} b{b} h{h}", exact_scores=True)
+            lock[(layer, b, h)] = ls
+    for t in range(S):
+        outs = {}
+        for layer in layers:
+            qd, kd, vd = dec[layer]
+            o = torch.empty_like(qd[t])
+            bz.decode_step(layer, qd[t], kd[t], vd[t], o)
+            outs[layer] = o
+        pre = {}
+        for key, ls in lock.items():
+            layer, b, h = key
+            qd, kd, vd = dec[layer]
+            ref = ls.decode(_np64(qd[t, b, h * g:(h + 1) * g]), _np64(kd[t, b, h]), _np64(vd[t, b, h]))
+            got = _np64(outs[layer][b, h * g:(h + 1) * g])
+            assert_close(got, ref, what=f"decode out step {t} {key}", **tol)
+            stats["max_out_err"] = max(stats["max_out_err"], float(np.abs(got - ref).max()))
+            will_evict = ls.counts()[0] >= w.budget
+            if will_evict or (t % check_every == 0) or t == S - 1:
+                st = compare_state(bz, ls, layer, b, h, f"decode step {t} {key}", exact_scores=False)
+                if will_evict:
+                    ls.set_scores(st["score"].numpy().astype(np.float64))
+            pre[key] = will_evict
+        for layer in layers:
+            bz.evict(layer)
+        assert bz.status() == 0, f"device status after step {t}"
+        for key, ls in lock.items():
+            r = ls.evict()
+            assert r == (1 if pre[key] else 0)
+            if pre[key]:
+                stats["evictions"] += 1
+                compare_state(bz, ls, *key, f"after eviction step {t} {key}", exact_scores=True)
+    if own:
+        bz.close()
+    return stats

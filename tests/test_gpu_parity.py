@@ -1,0 +1,230 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from oracle.buzz_oracle import OracleHead
+from tests.harness import (assert_close, assert_scores_close, compare_state, make_buzz, run_lockstep)
+
+pytestmark = pytest.mark.gpu
+
+
+def test_c1_full(cuda_device):
+    """The tiny fp32 workload in full: 512-token prompt, 256 decode steps, evictions on the way."""
+    w = workloads.get("C1")
+    stats = run_lockstep(w, [(0, 0, 0)])
+    assert stats["prefill_rounds"] == 1 and stats["evictions"] == 3
+
+
+def test_c2_shape_scaled(cuda_device):
+    """Llama-2-7B head shape (bf16, d=128, MHA), low-rank + outlier keys; several key tiles and a
+    ragged tail; budget small enough that decode-time evictions happen."""
+    w = workloads.scaled(workloads.get("C2"), layers=2, batch=3, q_heads=4, kv_heads=4,
+                         prompt_min=700, prompt_max=700, decode_steps=150, window=64, budget=180)
+    stats = run_lockstep(w, [(0, 0, 0), (0, 2, 3), (1, 1, 2)], check_every=7)
+    assert stats["prefill_rounds"] >= 1 and stats["evictions"] >= 3
+
+
+def test_c3_shape_scaled(cuda_device):
+    """Two hitters per segment of 16, AR(1) keys, prompt much longer than the budget."""
+    w = workloads.scaled(workloads.get("C3"), layers=1, batch=2, q_heads=2, kv_heads=2,
+                         prompt_min=1500, prompt_max=1500, decode_steps=200, window=96, budget=420)
+    stats = run_lockstep(w, [(0, 0, 1), (0, 1, 0)], check_every=9)
+    assert stats["evictions"] >= 2
+
+
+def test_c4_shape_scaled_gqa(cuda_device):
+    """Grouped-query attention: 4 query heads per KV head, scores summed over the group."""
+    w = workloads.scaled(workloads.get("C4"), layers=2, batch=2, q_heads=8, kv_heads=2,
+                         prompt_min=900, prompt_max=900, decode_steps=130, window=64, budget=300)
+    stats = run_lockstep(w, [(0, 1, 0), (1, 0, 1)], check_every=5)
+    assert stats["evictions"] >= 2
+
+
+def test_c5_shape_scaled_ragged(cuda_device):
+    """Ragged prompts, per-sequence eviction triggers."""
+    w = workloads.scaled(workloads.get("C5"), layers=1, batch=4, q_heads=2, kv_heads=2,
+                         prompt_min=300, prompt_max=900, decode_steps=180, window=48, budget=200)
+    lens = workloads.prompt_lengths(w)
+    assert len(set(lens)) > 1
+    stats = run_lockstep(w, [(0, b, b % 2) for b in range(4)], check_every=6)
+    assert stats["evictions"] >= 4
+
+
+def test_logn_scaling(cuda_device):
+    """log_512(n) logit scaling (Section 3.5) in prefill and decode."""
+    w = workloads.scaled(workloads.get("C1"), prompt_min=200, prompt_max=200, decode_steps=40)
+    run_lockstep(w, [(0, 0, 0)], logn=True)
+
+
+@pytest.mark.parametrize("N", [1, 3, 40, 68, 69, 159, 160, 161, 700])
+def test_prompt_length_edges(cuda_device, N):
+    """Prompts shorter than sink+window (Remark 1), just below / at / above the budget, and far
+    above it (Remark 2: several sampling rounds)."""
+    w = workloads.scaled(workloads.get("C1"), prompt_min=N, prompt_max=N, decode_steps=5,
+                         budget=160 if N < 700 else 84)
+    run_lockstep(w, [(0, 0, 0)])
+
+
+@pytest.mark.parametrize("dtype,d,g", [("bf16", 64, 1), ("bf16", 64, 2), ("f32", 128, 1), ("f32", 64, 4),
+                                       ("bf16", 128, 8)])
+def test_dtype_headdim_group_matrix(cuda_device, dtype, d, g):
+    w = workloads.scaled(workloads.get("C4"), layers=1, batch=2, q_heads=2 * g, kv_heads=2, head_dim=d,
+                         dtype=dtype, prompt_min=200, prompt_max=200, decode_steps=70, window=32,
+                         budget=128, segment=5, hitters=2)
+    stats = run_lockstep(w, [(0, 0, 0), (0, 1, 1)], check_every=3)
+    assert stats["evictions"] >= 2
+
+
+def _random_state(rng, n, d, dtype, quantum):
+    pos = np.sort(rng.choice(10 * n, size=n, replace=False)).astype(np.int32)
+    score = rng.random(n).astype(np.float32)
+    if quantum:
+        score = (np.round(score * quantum) / quantum).astype(np.float32)   # exact ties
+    k = torch.randn(n, d, generator=torch.Generator().manual_seed(int(rng.integers(1 << 30)))).to(dtype)
+    v = torch.randn(n, d, generator=torch.Generator().manual_seed(int(rng.integers(1 << 30)))).to(dtype)
+    return pos, score, k, v
+
+
+@pytest.mark.parametrize("segment,hitters,quantum", [(8, 1, 0), (8, 1, 4), (16, 2, 3), (5, 3, 2), (40, 7, 5),
+                                                    (3, 1, 2), (100, 33, 6)])
+def test_eviction_bit_exact_on_planted_states(cuda_device, segment, hitters, quantum):
+    """Planted cache states with exact score ties: indices, positions, scores and rows must match
+    the oracle bit for bit, for full caches with every possible n_old class and for caches below
+    the budget (which must be left alone)."""
+    rng = np.random.default_rng(segment * 131 + hitters)
+    sink, window, budget, d = 3, 17, 3 + 17 + 3 * segment + 57, 64
+    w = workloads.scaled(workloads.get("C1"), batch=6, q_heads=2, kv_heads=2, sink=sink, window=window,
+                         segment=segment, hitters=hitters, budget=budget, head_dim=d, dtype="bf16")
+    bz = make_buzz(w, max_prompt_tokens=64)
+    T = budget - sink - window
+    cases = []
+    for b in range(6):
+        for h in range(2):
+            n = budget if b < 5 else budget - 1 - h
+            n_old = [0, T, T // 2, 1, T - 1, 5][b]
+            n_old = min(n_old, n - sink - window)
+            pos, score, k, v = _random_state(rng, n, d, torch.bfloat16, quantum)
+            bz.import_state(0, b, h, n_old, int(pos[-1]) + 1, torch.from_numpy(pos), torch.from_numpy(score), k, v)
+            orc = OracleHead(1, d, sink, window, segment, hitters, budget)
+            orc.set_state(n_old, int(pos[-1]) + 1, pos, score.astype(np.float64), k.double().numpy(), v.double().numpy())
+            cases.append((b, h, orc, n))
+    bz.evict(0)
+    assert bz.status() == 0
+    for b, h, orc, n in cases:
+        r = orc.evict()
+        assert r == (1 if n >= budget else 0)
+        compare_state(bz, orc, 0, b, h, f"planted b{b} h{h}", exact_scores=True)
+    bz.evict(-1)                       # a second call must be a no-op everywhere
+    for b, h, orc, n in cases:
+        compare_state(bz, orc, 0, b, h, f"planted again b{b} h{h}", exact_scores=True)
+    bz.close()
+
+
+def test_decode_cluster_sizes_agree(cuda_device):
+    """The split of an instance over 1, 2, 4 or 8 CTAs changes only the fp32 summation order."""
+    w = workloads.scaled(workloads.get("C4"), layers=1, batch=2, q_heads=8, kv_heads=2,
+                         prompt_min=333, prompt_max=333, decode_steps=3, window=64, budget=400)
+    ref = None
+    for cs in (1, 2, 4, 8):
+        bz = make_buzz(w)
+        bz.set_decode_cluster(cs)
+        run_lockstep(w, [(0, 1, 1)], bz=bz)
+        st = bz.export_state(0, 1, 1)
+        if ref is None:
+            ref = st
+        else:
+            assert torch.equal(st["pos"], ref["pos"])
+            assert_scores_close(st["score"].numpy(), ref["score"].numpy(), f"cluster {cs}")
+        bz.close()
+
+
+def test_deterministic(cuda_device):
+    """Two runs on the same inputs give bit-identical caches and outputs."""
+    w = workloads.scaled(workloads.get("C2"), layers=1, batch=2, q_heads=2, kv_heads=2,
+                         prompt_min=500, prompt_max=500, decode_steps=90, window=32, budget=150)
+    snaps = []
+    for _ in range(2):
+        bz = make_buzz(w)
+        q, k, v, cu = workloads.prefill_inputs(w, 0, "cuda:0")
+        out = torch.empty_like(q)
+        bz.prefill(0, q, k, v, cu, 500, out)
+        qd, kd, vd = workloads.decode_inputs(w, 0, "cuda:0")
+        outs = [out.clone()]
+        for t in range(w.decode_steps):
+            o = torch.empty_like(qd[t])
+            bz.decode_step(0, qd[t], kd[t], vd[t], o)
+            bz.evict(0)
+            outs.append(o)
+        assert bz.status() == 0
+        snaps.append((outs, [bz.export_state(0, b, h) for b in range(2) for h in range(2)]))
+        bz.close()
+    for a, b in zip(snaps[0][0], snaps[1][0]):
+        assert torch.equal(a, b)
+    for a, b in zip(snaps[0][1], snaps[1][1]):
+        assert a["n"] == b["n"] and a["n_old"] == b["n_old"]
+        for key in ("pos", "score", "k", "v"):
+            assert torch.equal(a[key], b[key])
+
+
+def test_overflow_status(cuda_device):
+    w = workloads.scaled(workloads.get("C1"), prompt_min=100, prompt_max=100, budget=104, window=64)
+    bz = make_buzz(w)
+    q, k, v, cu = workloads.prefill_inputs(w, 0, "cuda:0")
+    bz.prefill(0, q, k, v, cu, 100, torch.empty_like(q))
+    qd, kd, vd = workloads.decode_inputs(w, 0, "cuda:0", steps=6)
+    o = torch.empty_like(qd[0])
+    for t in range(4):
+        bz.decode_step(0, qd[t], kd[t], vd[t], o)
+    assert bz.status() == 0 and bz.export_state(0, 0, 0)["n"] == 104
+    bz.decode_step(0, qd[4], kd[4], vd[4], o)          # cache full and no evict: must be refused
+    assert bz.status() == -2
+    assert bz.status() == 0                            # reading clears it
+    assert bz.export_state(0, 0, 0)["n"] == 104        # and the sequence was left untouched
+    bz.close()
+
+
+def test_no_progress_status(cuda_device):
+    """segment = 2 gives s_hat = 1: a cache full of old tokens cannot shrink; reported, not looped."""
+    w = workloads.scaled(workloads.get("C1"), sink=1, window=2, segment=2, hitters=1, budget=8,
+                         head_dim=64, dtype="f32")
+    bz = make_buzz(w, max_prompt_tokens=16)
+    n = 8
+    pos = torch.arange(n, dtype=torch.int32)
+    bz.import_state(0, 0, 0, n - 3, n, pos, torch.rand(n), torch.randn(n, 64), torch.randn(n, 64))
+    bz.evict(0)
+    assert bz.status() == -3
+    bz.close()
+
+
+def test_invalid_arguments_are_rejected(cuda_device):
+    from paper_2410_23079_b200 import Buzz, BuzzError
+    base = dict(sink=4, window=8, segment=4, hitters=1, budget=32, layers=1, max_batch=1, q_heads=2,
+                kv_heads=2, head_dim=64, dtype=torch.float32, max_prompt_tokens=64)
+    for bad in [dict(segment=1), dict(hitters=4), dict(window=0), dict(budget=15), dict(head_dim=96),
+                dict(q_heads=3), dict(sink=-1)]:
+        with pytest.raises(BuzzError):
+            Buzz(**{**base, **bad})
+    bz = Buzz(**base)
+    t = torch.zeros(64, 2, 64, device="cuda:0")
+    cu = torch.tensor([0, 64], dtype=torch.int32, device="cuda:0")
+    with pytest.raises(BuzzError):
+        bz.prefill(1, t, t, t, cu, 64, t)              # layer out of range
+    with pytest.raises(BuzzError):
+        bz.prefill(0, t[:1].expand(65, 2, 64), t, t, cu, 64, t)   # more tokens than sized for
+    bz.close()
+
+
+def test_full_size_c2_layer_sampled(cuda_device):
+    """One layer at the benchmark's full C2 shape (batch 8, 32 heads, 4096-token prompts, budget
+    1843), in the launch configuration bench.py times; the oracle checks three sampled instances,
+    and a conservation law checks every head: the prompt scores of a head sum to g * tokens."""
+    w = workloads.scaled(workloads.get("C2"), layers=1, decode_steps=3)
+    bz = make_buzz(w)
+    run_lockstep(w, [(0, 0, 0), (0, 7, 31), (0, 3, 17)], bz=bz)
+    total = w.batch * w.prompt_min
+    for h in range(0, w.kv_heads, 5):
+        s = bz.export_prefill_scores(h, total).double().sum().item()
+        assert abs(s - w.group * total) <= 1e-4 * total
+    bz.close()
