@@ -40,7 +40,8 @@ enum {
   BUZZ_ERR_OVERFLOW = -2,    /* decode step on a full cache (evict was not called in time)   */
   BUZZ_ERR_NO_PROGRESS = -3, /* an eviction left the cache full (degenerate parameters)      */
   BUZZ_ERR_TIMEOUT = -4,     /* a bounded on-device wait expired                             */
-  BUZZ_ERR_CUDA = -5         /* a CUDA runtime call failed                                   */
+  BUZZ_ERR_CUDA = -5,        /* a CUDA runtime call failed                                   */
+  BUZZ_ERR_TOO_LARGE = -6    /* request exceeds a built-in fixed-size buffer                 */
 };
 
 typedef struct buzz_ctx* buzz_t;
@@ -95,6 +96,30 @@ void buzz_destroy(buzz_t ctx);
 int buzz_prefill(buzz_t ctx, int layer, const void* q, const void* k, const void* v,
                  const int32_t* cu_seqlens_dev, int batch, int total_tokens, int max_seqlen,
                  void* out, void* stream);
+
+/* buzz_prefill for callers that cannot allocate device memory. (The paper has no counterpart;
+ * this is a property of the library, not of the method.)
+ * Some code runs where cudaMalloc is off limits: inside another framework's memory pool, in a
+ * real-time loop, in a process whose device memory was handed out once at start-up. Such a caller
+ * passes its inputs and outputs exactly as for buzz_prefill, and the prefill's temporaries (row
+ * softmax statistics and per-key column sums) are placed in a fixed 4 MiB array built into the
+ * library instead of in the scratch buffer given to buzz_create. Every GPU that loads the library
+ * holds that array until the process exits.
+ *   - Limit: (q_heads + kv_heads) * total_tokens <= BUZZ_STATIC_SCRATCH_FLOATS (1,048,576 floats);
+ *     larger calls return BUZZ_ERR_TOO_LARGE and launch nothing. total_tokens need not respect
+ *     max_prompt_tokens.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) with
+ *     that device current; make that first call outside any stream capture.
+ *   - The call allocates and frees nothing. All calls on a device share the array, which keeps
+ *     the previous call's contents (each call overwrites every entry before reading it, so no
+ *     clearing is needed); calls whose kernels overlap on the GPU race on it, so order them on
+ *     one stream or with events.
+ *   - buzz_export_prefill_scores does not see this call's scores (they are in the built-in array).
+ * Arguments, results, cache update and error behaviour are otherwise those of buzz_prefill. */
+#define BUZZ_STATIC_SCRATCH_FLOATS (1u << 20)
+int buzz_prefill_static(buzz_t ctx, int layer, const void* q, const void* k, const void* v,
+                        const int32_t* cu_seqlens_dev, int batch, int total_tokens, int max_seqlen,
+                        void* out, void* stream);
 
 /* One decode step of one layer (Eqs. 2 and 3) for the `batch` sequences of the last prefill:
  *   q [batch][Hq][d], k_new, v_new [batch][Hkv][d], out [batch][Hq][d].

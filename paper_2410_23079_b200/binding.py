@@ -36,7 +36,7 @@ def exported_symbols() -> list[str]:
     """Every entry point include/buzz.h declares."""
     return ["buzz_workspace_bytes", "buzz_create", "buzz_destroy", "buzz_prefill", "buzz_decode_step",
             "buzz_decode_step_host", "buzz_evict", "buzz_export_state", "buzz_import_state",
-            "buzz_export_prefill_scores",
+            "buzz_export_prefill_scores", "buzz_prefill_static",
             "buzz_status", "buzz_launch_count", "buzz_set_decode_cluster", "buzz_error_string"]
 
 
@@ -60,6 +60,8 @@ def load_library(build_if_missing: bool = True):
     lib.buzz_destroy.argtypes = [vp]
     lib.buzz_prefill.restype = ci
     lib.buzz_prefill.argtypes = [vp, ci, vp, vp, vp, vp, ci, ci, ci, vp, vp]
+    lib.buzz_prefill_static.restype = ci
+    lib.buzz_prefill_static.argtypes = [vp, ci, vp, vp, vp, vp, ci, ci, ci, vp, vp]
     lib.buzz_decode_step.restype = ci
     lib.buzz_decode_step.argtypes = [vp, ci, vp, vp, vp, vp, vp]
     lib.buzz_decode_step_host.restype = ci
@@ -148,6 +150,15 @@ class Buzz:
         _check(self._lib.buzz_prefill(self._h, layer, q.data_ptr(), k.data_ptr(), v.data_ptr(),
                                       cu_seqlens.data_ptr(), batch, q.shape[0], int(max_seqlen),
                                       out.data_ptr(), _stream_ptr(stream)), "buzz_prefill")
+
+    def prefill_static(self, layer, q, k, v, cu_seqlens, max_seqlen, out, stream=None):
+        """buzz_prefill_static: prefill whose temporaries live in the library's built-in 4 MiB device
+        array, for callers that must not allocate device memory. Same arguments as :meth:`prefill`;
+        raises BuzzError(-6) when (q_heads + kv_heads) * tokens exceeds 1,048,576 floats."""
+        batch = cu_seqlens.numel() - 1
+        _check(self._lib.buzz_prefill_static(self._h, layer, q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                             cu_seqlens.data_ptr(), batch, q.shape[0], int(max_seqlen),
+                                             out.data_ptr(), _stream_ptr(stream)), "buzz_prefill_static")
 
     def decode_step(self, layer, q, k_new, v_new, out, stream=None):
         _check(self._lib.buzz_decode_step(self._h, layer, q.data_ptr(), k_new.data_ptr(),

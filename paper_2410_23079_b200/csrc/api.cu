@@ -272,6 +272,7 @@ const char* buzz_error_string(int code) {
     case BUZZ_ERR_NO_PROGRESS: return "eviction cannot shrink the cache (segment too small for this budget)";
     case BUZZ_ERR_TIMEOUT: return "a bounded on-device wait expired";
     case BUZZ_ERR_CUDA: return "a CUDA runtime call failed";
+    case BUZZ_ERR_TOO_LARGE: return "request exceeds the library's built-in fixed-size scratch array";
     default: return "unknown error";
   }
 }
