@@ -25,7 +25,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int kUnroll = 4;      // 16-byte loads in flight per thread
+constexpr int kUnroll = 8;      // 16-byte loads in flight per thread
 constexpr int kMaxCluster = 8;
 
 template <typename T> struct Vec16;
@@ -336,11 +336,14 @@ cudaError_t buzz_launch_decode(buzz_ctx* c, int layer, const void* q, const void
   if (c->batch[layer] == 0) return cudaSuccess;
   int cs = c->decode_cluster;
   if (cs == 0) {
-    // Enough CTAs to fill 148 SMs several times over, chunks of at least ~64 rows.
+    // About three resident CTAs per SM (148 SMs) so that the whole grid is one wave: the smallest
+    // power-of-two split that gets there, while every CTA still streams at least ~64 rows.
     const long inst = (long)c->batch[layer] * c->sh.kv_heads;
     cs = 1;
-    while (cs < kMaxCluster && (c->pol.budget / (cs * 2)) >= 64 && inst * cs < 148L * 16) cs *= 2;
+    while (cs < kMaxCluster && inst * cs < 148L * 3 && (c->pol.budget / (cs * 2)) >= 64) cs *= 2;
   }
+  // the logits of a chunk must fit in shared memory
+  while (cs < kMaxCluster && (size_t)c->group * ((c->pol.budget + cs - 1) / cs) * sizeof(float) > 96 * 1024) cs *= 2;
   cudaError_t e;
   if (c->sh.dtype == BUZZ_BF16) {
     e = c->sh.head_dim == 128 ? launch_g<__nv_bfloat16, 128>(c, layer, q, k_new, v_new, out, cs, stream)
