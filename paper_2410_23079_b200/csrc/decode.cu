@@ -331,23 +331,26 @@ cudaError_t launch_g(buzz_ctx* c, int layer, const void* q, const void* k_new, c
 
 }  // namespace
 
+cudaError_t buzz_launch_decode_bf16(buzz_ctx* c, int layer, const void* q, const void* k_new,
+                                    const void* v_new, void* out, int cluster_size, cudaStream_t stream);
+
 cudaError_t buzz_launch_decode(buzz_ctx* c, int layer, const void* q, const void* k_new,
                                const void* v_new, void* out, cudaStream_t stream) {
   if (c->batch[layer] == 0) return cudaSuccess;
   int cs = c->decode_cluster;
   if (cs == 0) {
-    // About three resident CTAs per SM (148 SMs) so that the whole grid is one wave: the smallest
-    // power-of-two split that gets there, while every CTA still streams at least ~64 rows.
+    // The whole grid should be one resident wave of long-lived CTAs: the smallest power-of-two
+    // split that gives every one of the 148 SMs at least one or two CTAs (measured best on C2 and
+    // C4 shapes), while every CTA still streams at least ~64 rows.
     const long inst = (long)c->batch[layer] * c->sh.kv_heads;
     cs = 1;
-    while (cs < kMaxCluster && inst * cs < 148L * 3 && (c->pol.budget / (cs * 2)) >= 64) cs *= 2;
+    while (cs < kMaxCluster && inst * cs < 148L * 3 / 2 && (c->pol.budget / (cs * 2)) >= 64) cs *= 2;
   }
   // the logits of a chunk must fit in shared memory
   while (cs < kMaxCluster && (size_t)c->group * ((c->pol.budget + cs - 1) / cs) * sizeof(float) > 96 * 1024) cs *= 2;
   cudaError_t e;
   if (c->sh.dtype == BUZZ_BF16) {
-    e = c->sh.head_dim == 128 ? launch_g<__nv_bfloat16, 128>(c, layer, q, k_new, v_new, out, cs, stream)
-                              : launch_g<__nv_bfloat16, 64>(c, layer, q, k_new, v_new, out, cs, stream);
+    e = buzz_launch_decode_bf16(c, layer, q, k_new, v_new, out, cs, stream);   // tensor-core kernel
   } else {
     e = c->sh.head_dim == 128 ? launch_g<float, 128>(c, layer, q, k_new, v_new, out, cs, stream)
                               : launch_g<float, 64>(c, layer, q, k_new, v_new, out, cs, stream);
