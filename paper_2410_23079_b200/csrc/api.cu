@@ -10,6 +10,10 @@ cudaError_t buzz_launch_prefill_simt(buzz_ctx* c, const void* q, const void* k, 
                                      const int32_t* cu, int batch, int max_seqlen, void* out,
                                      cudaStream_t stream, int* launches);
 
+cudaError_t buzz_launch_prefill_tc(buzz_ctx* c, const void* q, const void* k, const void* v,
+                                   const int32_t* cu, int batch, int total_tokens, int max_seqlen,
+                                   void* out, cudaStream_t stream, int* launches);
+
 namespace {
 
 constexpr size_t kAlign = 256;
@@ -136,7 +140,10 @@ int buzz_prefill(buzz_t c, int layer, const void* q, const void* k, const void* 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int launches = 0;
   cudaError_t e;
-  e = buzz_launch_prefill_simt(c, q, k, v, cu_seqlens_dev, batch, max_seqlen, out, s, &launches);
+  if (c->sh.dtype == BUZZ_BF16 && c->sh.head_dim == 128)   // tensor-core path (TMA + tcgen05 + TMEM)
+    e = buzz_launch_prefill_tc(c, q, k, v, cu_seqlens_dev, batch, total_tokens, max_seqlen, out, s, &launches);
+  else
+    e = buzz_launch_prefill_simt(c, q, k, v, cu_seqlens_dev, batch, max_seqlen, out, s, &launches);
   c->launches += launches;
   if (e != cudaSuccess) return BUZZ_ERR_CUDA;
   c->batch[layer] = batch;

@@ -1,0 +1,457 @@
+// Prefill attention with per-key column sums for bf16, head_dim 128, on the Blackwell tensor
+// cores: TMA-fed tcgen05 MMAs with accumulators in tensor memory (TMEM).
+//
+// What is computed (Eqs. 1 and 3 of the paper, and Algorithm 2's accumulated attention A):
+//   O = Softmax(Q K^T / sqrt(d)) V, causal, per sequence and query head, and for every key j
+//   score_j = sum over the group's query heads and rows i >= j of P_ij.
+// The column sums need each row's FINAL normaliser, so S = Q K^T is formed twice:
+//   pass A  (attn_tc_kernel, query-tile stationary) flash-style attention: S in TMEM, one thread
+//           per row does the online softmax, P goes back to TMEM as bf16 and is the A operand of
+//           the P V MMA; the output accumulator lives in TMEM and is rescaled lazily (only when a
+//           row maximum grows by more than 2^8). Writes O and the row log2-sum-exp.
+//   pass B  (colsum_tc_kernel, key-tile stationary) S^T = K Q^T in TMEM with KEYS on the TMEM
+//           lanes, so one thread owns one key: it forms the exact probabilities 2^(S - lse) in
+//           fp32 and adds them up over the query rows in a fixed order (heads, then tiles, then
+//           rows ascending) -- no cross-thread reduction, no atomics, bit-reproducible.
+// Warp roles in both kernels: warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM owner),
+// warps 2..5 = one thread per TMEM lane. All mbarrier waits are bounded; a wait that gives up sets
+// BUZZ_ERR_TIMEOUT and the CTA runs to its end without touching more data.
+#include <math.h>
+
+#include "buzz_internal.cuh"
+#include "sm100_ptx.cuh"
+
+namespace {
+
+using namespace sm100;
+
+constexpr int D = 128;                    // head dim
+constexpr int BT = 128;                   // tile edge: query rows and keys per tile
+constexpr int kThreads = 192;
+constexpr uint32_t kBlockBytes = BT * 128;          // one [128 rows x 64 bf16] swizzled block
+constexpr uint32_t kTileBytes = 2 * kBlockBytes;    // a [128 x 128] bf16 tile = two blocks
+constexpr float kInvLn512 = 1.0f / 6.2383246250395077f;
+constexpr uint32_t kIdescKK = idesc_bf16(BT, BT, false, false);   // both operands K-major
+constexpr uint32_t kIdescKM = idesc_bf16(BT, BT, false, true);    // B operand MN-major (V)
+
+struct TimeoutFlag {
+  int32_t* status;
+  int inst;
+  __device__ void raise(int where) const { buzz_set_status(status, BUZZ_ERR_TIMEOUT, inst, where); }
+};
+
+// K-major operand tile ([rows][128 dims] as two swizzled blocks): descriptor of k-step ks (16 dims).
+__device__ __forceinline__ uint64_t kmajor_desc(uint32_t tile_saddr, int ks) {
+  return smem_desc_sw128(tile_saddr + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024);
+}
+// MN-major operand tile (V: [keys][128 dims]): descriptor of k-step ks (16 keys), N = 128 dims.
+__device__ __forceinline__ uint64_t mnmajor_desc(uint32_t tile_saddr, int ks) {
+  return smem_desc_sw128(tile_saddr + ks * 16 * 128, kBlockBytes, 1024);
+}
+
+// One [128 x 128] bf16 tile = two TMA boxes of 64 columns.
+__device__ __forceinline__ void load_tile(void* dst, const CUtensorMap* map, int col0, int row0, uint64_t* bar) {
+  tma_load_2d(dst, map, col0, row0, bar);
+  tma_load_2d(static_cast<char*>(dst) + kBlockBytes, map, col0 + 64, row0, bar);
+}
+
+// =================================================================================================
+// Pass B: column sums. grid (key tiles, kv heads, sequences), 2 CTAs per SM.
+// =================================================================================================
+struct SmemB {
+  alignas(1024) unsigned char k[kTileBytes];
+  alignas(1024) unsigned char q[2][kTileBytes];
+  float lse[2][BT];
+  float rs[2][BT];
+  uint64_t k_full, q_full[2], q_empty[2], s_full[2], s_empty[2];
+  uint32_t tmem_base;
+};
+
+__global__ void __launch_bounds__(kThreads, 2)
+colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                 const int32_t* __restrict__ cu, const float* __restrict__ lse, float* __restrict__ pscore,
+                 int32_t* status, int Hq, int Hkv, int stride, float scale_log2, int logn) {
+  extern __shared__ unsigned char smem_raw[];
+  SmemB& sm = *reinterpret_cast<SmemB*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int b = blockIdx.z, kvh = blockIdx.y, G = Hq / Hkv;
+  const int tok0 = cu[b], N = cu[b + 1] - tok0;
+  const int kt = blockIdx.x, key0 = kt * BT;
+  if (key0 >= N) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q_tiles = (N + BT - 1) / BT;
+  const int nq = q_tiles - kt;
+  const int iters = G * nq;
+  const TimeoutFlag tf{status, (b * Hkv + kvh) * 4096 + kt};
+
+  if (threadIdx.x == 0) {
+    mbar_init(&sm.k_full, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sm.q_full[s], 1);
+      mbar_init(&sm.q_empty[s], 1);
+      mbar_init(&sm.s_full[s], 1);
+      mbar_init(&sm.s_empty[s], 128);
+    }
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&sm.tmem_base, 256);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sm.tmem_base;
+
+  if (warp == 0) {
+    // ---- TMA producer ----
+    if (elect_one()) {
+      prefetch_tensormap(&map_q);
+      prefetch_tensormap(&map_k);
+      mbar_expect_tx(&sm.k_full, kTileBytes);
+      load_tile(sm.k, &map_k, kvh * D, tok0 + key0, &sm.k_full);
+      for (int it = 0; it < iters; ++it) {
+        const int st = it & 1, use = it >> 1;
+        if (use > 0 && !mbar_wait(&sm.q_empty[st], (use - 1) & 1)) { tf.raise(1); break; }
+        const int g = it / nq, qt = kt + it % nq;
+        mbar_expect_tx(&sm.q_full[st], kTileBytes);
+        load_tile(sm.q[st], &map_q, (kvh * G + g) * D, tok0 + qt * BT, &sm.q_full[st]);
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer: S^T[keys x rows] = K Q^T ----
+    if (elect_one()) {
+      bool ok = mbar_wait(&sm.k_full, 0);
+      if (!ok) tf.raise(2);
+      for (int it = 0; ok && it < iters; ++it) {
+        const int st = it & 1, use = it >> 1;
+        if (!mbar_wait(&sm.q_full[st], use & 1)) { tf.raise(3); break; }
+        if (use > 0 && !mbar_wait(&sm.s_empty[st], (use - 1) & 1)) { tf.raise(4); break; }
+        tc_fence_after();
+        const uint32_t ka = smem_u32(sm.k), qa = smem_u32(sm.q[st]);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks)
+          mma_ss(tmem + st * BT, kmajor_desc(ka, ks), kmajor_desc(qa, ks), kIdescKK, ks > 0);
+        mma_commit(&sm.s_full[st]);
+        mma_commit(&sm.q_empty[st]);
+      }
+    }
+  } else {
+    // ---- one thread per key: exact probabilities, summed down the column ----
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;              // TMEM lane = key within the tile
+    const int t = (warp - 2) * 32 + lane;             // 0..127 among the compute threads
+    const int kpos = key0 + row;
+    float colsum = 0.f;
+    for (int it = 0; it < iters; ++it) {
+      const int st = it & 1, use = it >> 1;
+      const int g = it / nq, qt = kt + it % nq;
+      const int q0 = qt * BT;
+      const int h = kvh * G + g;
+      // stage this tile's row statistics; the named barrier below publishes them
+      {
+        const int qpos = q0 + t;
+        sm.lse[st][t] = (qpos < N) ? lse[(size_t)h * stride + tok0 + qpos] : 0.f;
+        sm.rs[st][t] = scale_log2 * (logn ? __logf((float)(qpos + 1)) * kInvLn512 : 1.0f);
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (!mbar_wait(&sm.s_full[st], use & 1)) { tf.raise(5); break; }
+      tc_fence_after();
+      const bool diag = (qt == kt), tail = (q0 + BT > N);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BT; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + st * BT + c0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const float p = exp2f(__uint_as_float(r[c]) * sm.rs[st][c0 + c] - sm.lse[st][c0 + c]);
+          const int qpos = q0 + c0 + c;
+          const bool on = (!diag || qpos >= kpos) && (!tail || qpos < N);
+          colsum += on ? p : 0.f;
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(&sm.s_empty[st]);
+      // lse[st]/rs[st] are restaged two iterations from now; the named barrier of the next
+      // iteration, which every thread reaches only after these reads, orders that.
+    }
+    if (kpos < N) pscore[(size_t)kvh * stride + tok0 + kpos] = colsum;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 256);
+  }
+}
+
+// =================================================================================================
+// Pass A: attention output and row log-sum-exp. grid (query tiles, query heads, sequences), 1 CTA/SM.
+// TMEM columns: S0 [0,128)  S1 [128,256)  O [256,384); P (bf16 pairs) overwrites the first 64
+// columns of the S buffer it was computed from.
+// =================================================================================================
+struct SmemA {
+  alignas(1024) unsigned char q[kTileBytes];
+  alignas(1024) unsigned char k[3][kTileBytes];
+  alignas(1024) unsigned char v[2][kTileBytes];
+  uint64_t q_full, k_full[3], k_empty[3], v_full[2], v_empty[2], s_full[2], p_full[2], o_done;
+  uint32_t tmem_base;
+};
+constexpr uint32_t kColO = 256;
+constexpr float kRescaleThreshold = 8.0f;     // log2: rescale O only when a row max grows by > 2^8
+
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+               const __grid_constant__ CUtensorMap map_v, const int32_t* __restrict__ cu,
+               __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int32_t* status, int Hq, int Hkv,
+               int stride, float scale_log2, int logn) {
+  extern __shared__ unsigned char smem_raw[];
+  SmemA& sm = *reinterpret_cast<SmemA*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int b = blockIdx.z, h = blockIdx.y, kvh = h / (Hq / Hkv);
+  const int tok0 = cu[b], N = cu[b + 1] - tok0;
+  const int qt = gridDim.x - 1 - blockIdx.x;          // heaviest (last) query tiles first
+  const int row0 = qt * BT;
+  if (row0 >= N) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nt = qt + 1;                              // key tiles 0..qt (causal)
+  const TimeoutFlag tf{status, (b * Hq + h) * 4096 + qt};
+
+  if (threadIdx.x == 0) {
+    mbar_init(&sm.q_full, 1);
+    for (int s = 0; s < 3; ++s) { mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
+      mbar_init(&sm.s_full[s], 1); mbar_init(&sm.p_full[s], 128);
+    }
+    mbar_init(&sm.o_done, 1);
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&sm.tmem_base, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sm.tmem_base;
+
+  if (warp == 0) {
+    // ---- TMA producer ----
+    if (elect_one()) {
+      prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
+      mbar_expect_tx(&sm.q_full, kTileBytes);
+      load_tile(sm.q, &map_q, h * D, tok0 + row0, &sm.q_full);
+      for (int j = 0; j < nt; ++j) {
+        const int ks = j % 3, ku = j / 3, vs = j & 1, vu = j >> 1;
+        if (ku > 0 && !mbar_wait(&sm.k_empty[ks], (ku - 1) & 1)) { tf.raise(11); break; }
+        mbar_expect_tx(&sm.k_full[ks], kTileBytes);
+        load_tile(sm.k[ks], &map_k, kvh * D, tok0 + j * BT, &sm.k_full[ks]);
+        if (vu > 0 && !mbar_wait(&sm.v_empty[vs], (vu - 1) & 1)) { tf.raise(12); break; }
+        mbar_expect_tx(&sm.v_full[vs], kTileBytes);
+        load_tile(sm.v[vs], &map_v, kvh * D, tok0 + j * BT, &sm.v_full[vs]);
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer ----
+    if (elect_one()) {
+      const uint32_t qa = smem_u32(sm.q);
+      auto issue_qk = [&](int j) -> bool {             // S[j%2] = Q K_j^T
+        const int ks = j % 3;
+        if (!mbar_wait(&sm.k_full[ks], (j / 3) & 1)) { tf.raise(13); return false; }
+        tc_fence_after();
+        const uint32_t ka = smem_u32(sm.k[ks]);
+#pragma unroll
+        for (int s = 0; s < D / 16; ++s)
+          mma_ss(tmem + (j & 1) * BT, kmajor_desc(qa, s), kmajor_desc(ka, s), kIdescKK, s > 0);
+        mma_commit(&sm.s_full[j & 1]);
+        mma_commit(&sm.k_empty[ks]);
+        return true;
+      };
+      bool ok = mbar_wait(&sm.q_full, 0);
+      if (!ok) tf.raise(14);
+      ok = ok && issue_qk(0);
+      for (int j = 0; ok && j < nt; ++j) {
+        if (j + 1 < nt && !issue_qk(j + 1)) break;     // next tile's logits overlap this tile's softmax
+        const int sb = j & 1, use = j >> 1;
+        if (!mbar_wait(&sm.p_full[sb], use & 1)) { tf.raise(15); break; }
+        if (!mbar_wait(&sm.v_full[sb], use & 1)) { tf.raise(16); break; }
+        tc_fence_after();
+        const uint32_t va = smem_u32(sm.v[sb]);
+#pragma unroll
+        for (int s = 0; s < BT / 16; ++s)              // O += P_j V_j, 16 keys per step
+          mma_ts(tmem + kColO, tmem + sb * BT + s * 8, mnmajor_desc(va, s), kIdescKM, (j > 0 || s > 0) ? 1u : 0u);
+        mma_commit(&sm.v_empty[sb]);
+        mma_commit(&sm.o_done);
+      }
+    }
+  } else {
+    // ---- softmax: one thread per query row ----
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int qpos = row0 + row;
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const float rs = scale_log2 * (logn ? __logf((float)(qpos + 1)) * kInvLn512 : 1.0f);
+    float m_used = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < nt; ++j) {
+      const int sb = j & 1, use = j >> 1;
+      if (!mbar_wait(&sm.s_full[sb], use & 1)) { tf.raise(17); ok = false; break; }
+      tc_fence_after();
+      float s[BT];
+#pragma unroll
+      for (int c0 = 0; c0 < BT; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem + lane_base + sb * BT + c0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) s[c0 + c] = __uint_as_float(r[c]) * rs;
+      }
+      if (j == nt - 1) {                               // the diagonal tile: causal mask
+#pragma unroll
+        for (int c = 0; c < BT; ++c)
+          if (j * BT + c > qpos) s[c] = -INFINITY;
+      }
+      float mx = s[0];
+#pragma unroll
+      for (int c = 1; c < BT; ++c) mx = fmaxf(mx, s[c]);
+      const float m_new = fmaxf(m_used, mx);
+      if (j == 0) {
+        m_used = m_new;
+      } else {
+        const bool need = m_new > m_used + kRescaleThreshold;
+        if (__any_sync(0xffffffffu, need)) {            // rare after the first tiles
+          const float alpha = need ? exp2f(m_used - m_new) : 1.0f;
+          if (need) m_used = m_new;
+          l *= alpha;
+          if (!mbar_wait(&sm.o_done, (j - 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
+          tc_fence_after();
+#pragma unroll 1
+          for (int c0 = 0; c0 < D; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(tmem + lane_base + kColO + c0, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
+            tmem_st32(tmem + lane_base + kColO + c0, r);
+          }
+          tmem_wait_st();
+        }
+      }
+      // P = 2^(S - m) as bf16 pairs into the first 64 columns of this S buffer
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        uint32_t pk[32];
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const float p0 = exp2f(s[half * 64 + 2 * c] - m_used);
+          const float p1 = exp2f(s[half * 64 + 2 * c + 1] - m_used);
+          l += p0 + p1;
+          const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
+          pk[c] = *reinterpret_cast<const uint32_t*>(&pp);
+        }
+        tmem_st32(tmem + lane_base + sb * BT + half * 32, pk);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&sm.p_full[sb]);
+    }
+    // ---- epilogue: O / l -> bf16, row log2-sum-exp ----
+    if (ok && mbar_wait(&sm.o_done, (nt - 1) & 1)) {
+      tc_fence_after();
+      const float inv = 1.0f / l;
+      __nv_bfloat16* orow = out + ((size_t)(tok0 + qpos) * Hq + h) * D;
+#pragma unroll 1
+      for (int c0 = 0; c0 < D; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem + lane_base + kColO + c0, r);
+        tmem_wait_ld();
+        if (qpos < N) {
+#pragma unroll
+          for (int c = 0; c < 32; c += 8) {
+            uint4 o;
+            __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(r[c]) * inv, __uint_as_float(r[c + 1]) * inv);
+            __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(r[c + 2]) * inv, __uint_as_float(r[c + 3]) * inv);
+            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(r[c + 4]) * inv, __uint_as_float(r[c + 5]) * inv);
+            __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(r[c + 6]) * inv, __uint_as_float(r[c + 7]) * inv);
+            o.x = *reinterpret_cast<uint32_t*>(&t0); o.y = *reinterpret_cast<uint32_t*>(&t1);
+            o.z = *reinterpret_cast<uint32_t*>(&t2); o.w = *reinterpret_cast<uint32_t*>(&t3);
+            *reinterpret_cast<uint4*>(orow + c0 + c) = o;
+          }
+        }
+      }
+      if (qpos < N) lse[(size_t)h * stride + tok0 + qpos] = m_used + log2f(l);
+    } else if (ok) {
+      tf.raise(19);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// ---- host side --------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [tokens][heads * 128] bf16, boxes of 64 columns x 128 rows, 128-byte swizzle, zero fill out of range.
+bool make_map(CUtensorMap* map, const void* base, int tokens, int heads) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)heads * D, (cuuint64_t)tokens};
+  const cuuint64_t strides[1] = {(cuuint64_t)heads * D * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)BT};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t buzz_launch_prefill_tc(buzz_ctx* c, const void* q, const void* k, const void* v,
+                                   const int32_t* cu, int batch, int total_tokens, int max_seqlen,
+                                   void* out, cudaStream_t stream, int* launches) {
+  CUtensorMap mq, mk, mv;
+  if (!make_map(&mq, q, total_tokens, c->sh.q_heads) || !make_map(&mk, k, total_tokens, c->sh.kv_heads) ||
+      !make_map(&mv, v, total_tokens, c->sh.kv_heads))
+    return cudaErrorInvalidValue;
+  const size_t smemA = sizeof(SmemA) + 1024, smemB = sizeof(SmemB) + 1024;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smemA);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smemB);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  const int tiles = (max_seqlen + BT - 1) / BT;
+  const float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
+  const int logn = (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0;
+  attn_tc_kernel<<<dim3(tiles, c->sh.q_heads, batch), kThreads, smemA, stream>>>(
+      mq, mk, mv, cu, (__nv_bfloat16*)out, c->lse, c->st.status, c->sh.q_heads, c->sh.kv_heads,
+      c->sh.max_prompt_tokens, scale_log2, logn);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  colsum_tc_kernel<<<dim3(tiles, c->sh.kv_heads, batch), kThreads, smemB, stream>>>(
+      mq, mk, cu, c->lse, c->pscore, c->st.status, c->sh.q_heads, c->sh.kv_heads, c->sh.max_prompt_tokens,
+      scale_log2, logn);
+  *launches += 2;
+  return cudaGetLastError();
+}
