@@ -55,6 +55,29 @@ __device__ __forceinline__ void load_tile(void* dst, const CUtensorMap* map, int
   tma_load_2d(static_cast<char*>(dst) + kBlockBytes, map, col0 + 64, row0, bar);
 }
 
+// One key's 128 logits against one query tile -> exact probabilities added into four interleaved
+// accumulators (column c -> acc[c % 4]), so the summation order is fixed and the adds pipeline.
+template <bool LOGN>
+__device__ __forceinline__ void colsum_tile(const uint32_t (&r)[BT], const float* __restrict__ rs,
+                                            const float* __restrict__ lse, float scale_log2, bool diag,
+                                            bool tail, int q0, int kpos, int N, float (&acc)[4]) {
+  if (!diag && !tail) {
+#pragma unroll
+    for (int c = 0; c < BT; ++c) {
+      const float sc = LOGN ? rs[c] : scale_log2;
+      acc[c & 3] += exp2f(fmaf(__uint_as_float(r[c]), sc, -lse[c]));
+    }
+  } else {
+#pragma unroll
+    for (int c = 0; c < BT; ++c) {
+      const float sc = LOGN ? rs[c] : scale_log2;
+      const float p = exp2f(fmaf(__uint_as_float(r[c]), sc, -lse[c]));
+      const int qpos = q0 + c;
+      acc[c & 3] += (qpos >= kpos && qpos < N) ? p : 0.f;
+    }
+  }
+}
+
 // =================================================================================================
 // Pass B: column sums. grid (key tiles, kv heads, sequences), 2 CTAs per SM.
 // =================================================================================================
@@ -141,7 +164,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int row = quarter * 32 + lane;              // TMEM lane = key within the tile
     const int t = (warp - 2) * 32 + lane;             // 0..127 among the compute threads
     const int kpos = key0 + row;
-    float colsum = 0.f;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};           // column c adds into acc[c % 4]: a fixed order
     for (int it = 0; it < iters; ++it) {
       const int st = it & 1, use = it >> 1;
       const int g = it / nq, qt = kt + it % nq;
@@ -157,25 +180,21 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (!mbar_wait(&sm.s_full[st], use & 1)) { tf.raise(5); break; }
       tc_fence_after();
       const bool diag = (qt == kt), tail = (q0 + BT > N);
-#pragma unroll 1
-      for (int c0 = 0; c0 < BT; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + st * BT + c0, r);
-        tmem_wait_ld();
+      // the whole row of S^T first (four loads in flight), then 128 independent exponentials
+      uint32_t r[BT];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          const float p = exp2f(__uint_as_float(r[c]) * sm.rs[st][c0 + c] - sm.lse[st][c0 + c]);
-          const int qpos = q0 + c0 + c;
-          const bool on = (!diag || qpos >= kpos) && (!tail || qpos < N);
-          colsum += on ? p : 0.f;
-        }
-      }
+      for (int c0 = 0; c0 < BT; c0 += 32)
+        tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + st * BT + c0, *reinterpret_cast<uint32_t(*)[32]>(&r[c0]));
+      tmem_wait_ld();
       tc_fence_before();
-      mbar_arrive(&sm.s_empty[st]);
+      mbar_arrive(&sm.s_empty[st]);                    // S^T[st] may be overwritten from here on
+      if (logn) colsum_tile<true>(r, sm.rs[st], sm.lse[st], scale_log2, diag, tail, q0, kpos, N, acc);
+      else colsum_tile<false>(r, sm.rs[st], sm.lse[st], scale_log2, diag, tail, q0, kpos, N, acc);
+
       // lse[st]/rs[st] are restaged two iterations from now; the named barrier of the next
       // iteration, which every thread reaches only after these reads, orders that.
     }
-    if (kpos < N) pscore[(size_t)kvh * stride + tok0 + kpos] = colsum;
+    if (kpos < N) pscore[(size_t)kvh * stride + tok0 + kpos] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
   }
   tc_fence_before();
   __syncthreads();
@@ -187,17 +206,19 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
 // =================================================================================================
 // Pass A: attention output and row log-sum-exp. grid (query tiles, query heads, sequences), 1 CTA/SM.
-// TMEM columns: S0 [0,128)  S1 [128,256)  O [256,384); P (bf16 pairs) overwrites the first 64
-// columns of the S buffer it was computed from.
+// TMEM columns: S0 [0,128)  S1 [128,256)  P0 [256,320)  P1 [320,384) (bf16 pairs)  O [384,512).
+// P has buffers of its own: the tensor core may still be reading P of tile j-1 as the A operand
+// while the logits of tile j+1 are being written, so it must not share columns with S.
 // =================================================================================================
 struct SmemA {
   alignas(1024) unsigned char q[kTileBytes];
   alignas(1024) unsigned char k[3][kTileBytes];
   alignas(1024) unsigned char v[2][kTileBytes];
-  uint64_t q_full, k_full[3], k_empty[3], v_full[2], v_empty[2], s_full[2], p_full[2], o_done;
+  uint64_t q_full, k_full[3], k_empty[3], v_full[2], v_empty[2], s_full[2], p_full[2], o_done[2];
   uint32_t tmem_base;
 };
-constexpr uint32_t kColO = 256;
+constexpr uint32_t kColP = 256;
+constexpr uint32_t kColO = 384;
 constexpr float kRescaleThreshold = 8.0f;     // log2: rescale O only when a row max grows by > 2^8
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -223,7 +244,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
       mbar_init(&sm.s_full[s], 1); mbar_init(&sm.p_full[s], 128);
     }
-    mbar_init(&sm.o_done, 1);
+    mbar_init(&sm.o_done[0], 1);
+    mbar_init(&sm.o_done[1], 1);
     fence_barrier_init();
   }
   if (warp == 1) {
@@ -279,9 +301,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const uint32_t va = smem_u32(sm.v[sb]);
 #pragma unroll
         for (int s = 0; s < BT / 16; ++s)              // O += P_j V_j, 16 keys per step
-          mma_ts(tmem + kColO, tmem + sb * BT + s * 8, mnmajor_desc(va, s), kIdescKM, (j > 0 || s > 0) ? 1u : 0u);
+          mma_ts(tmem + kColO, tmem + kColP + sb * 64 + s * 8, mnmajor_desc(va, s), kIdescKM, (j > 0 || s > 0) ? 1u : 0u);
         mma_commit(&sm.v_empty[sb]);
-        mma_commit(&sm.o_done);
+        mma_commit(&sm.o_done[sb]);
       }
     }
   } else {
@@ -297,23 +319,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const int sb = j & 1, use = j >> 1;
       if (!mbar_wait(&sm.s_full[sb], use & 1)) { tf.raise(17); ok = false; break; }
       tc_fence_after();
+      // the raw logits of this row (rs > 0, so the row maximum can be taken before scaling)
       float s[BT];
 #pragma unroll
-      for (int c0 = 0; c0 < BT; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(tmem + lane_base + sb * BT + c0, r);
-        tmem_wait_ld();
-#pragma unroll
-        for (int c = 0; c < 32; ++c) s[c0 + c] = __uint_as_float(r[c]) * rs;
-      }
+      for (int c0 = 0; c0 < BT; c0 += 32)
+        tmem_ld32(tmem + lane_base + sb * BT + c0, *reinterpret_cast<uint32_t(*)[32]>(&s[c0]));
+      tmem_wait_ld();
       if (j == nt - 1) {                               // the diagonal tile: causal mask
 #pragma unroll
         for (int c = 0; c < BT; ++c)
           if (j * BT + c > qpos) s[c] = -INFINITY;
       }
-      float mx = s[0];
+      float mx4[4] = {s[0], s[1], s[2], s[3]};
 #pragma unroll
-      for (int c = 1; c < BT; ++c) mx = fmaxf(mx, s[c]);
+      for (int c = 4; c < BT; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], s[c]);
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * rs;
       const float m_new = fmaxf(m_used, mx);
       if (j == 0) {
         m_used = m_new;
@@ -323,7 +343,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           const float alpha = need ? exp2f(m_used - m_new) : 1.0f;
           if (need) m_used = m_new;
           l *= alpha;
-          if (!mbar_wait(&sm.o_done, (j - 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
+          if (!mbar_wait(&sm.o_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
           tc_fence_after();
 #pragma unroll 1
           for (int c0 = 0; c0 < D; c0 += 32) {
@@ -337,26 +357,30 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           tmem_wait_st();
         }
       }
-      // P = 2^(S - m) as bf16 pairs into the first 64 columns of this S buffer
+      // P = 2^(S rs - m) as bf16 pairs into P[sb], once the P V product of tile j-2 has consumed it
+      if (j >= 2 && !mbar_wait(&sm.o_done[sb], ((j >> 1) - 1) & 1)) { tf.raise(20); ok = false; break; }
+      const float neg_m = -m_used;
+      float l4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         uint32_t pk[32];
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
-          const float p0 = exp2f(s[half * 64 + 2 * c] - m_used);
-          const float p1 = exp2f(s[half * 64 + 2 * c + 1] - m_used);
-          l += p0 + p1;
+          const float p0 = exp2f(fmaf(s[half * 64 + 2 * c], rs, neg_m));
+          const float p1 = exp2f(fmaf(s[half * 64 + 2 * c + 1], rs, neg_m));
+          l4[c & 3] += p0 + p1;
           const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
           pk[c] = *reinterpret_cast<const uint32_t*>(&pp);
         }
-        tmem_st32(tmem + lane_base + sb * BT + half * 32, pk);
+        tmem_st32(tmem + lane_base + kColP + sb * 64 + half * 32, pk);
       }
+      l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&sm.p_full[sb]);
     }
     // ---- epilogue: O / l -> bf16, row log2-sum-exp ----
-    if (ok && mbar_wait(&sm.o_done, (nt - 1) & 1)) {
+    if (ok && mbar_wait(&sm.o_done[(nt - 1) & 1], ((nt - 1) >> 1) & 1)) {
       tc_fence_after();
       const float inv = 1.0f / l;
       __nv_bfloat16* orow = out + ((size_t)(tok0 + qpos) * Hq + h) * D;
