@@ -39,6 +39,27 @@ def _peaks():
     return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
 
 
+def _ncu_traffic(slots_per_launch):
+    """DRAM bytes per launch of the decode kernel from the committed ncu capture, scaled by the slots
+    one launch processes; None if there is no capture or the kernel source changed since it."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.txt")
+    if slots_per_launch is None or not os.path.exists(path):
+        return None
+    kv = {}
+    for line in open(path):
+        if "=" in line and not line.startswith("#"):
+            a, b = line.split("=", 1)
+            kv[a.strip()] = b.strip()
+    try:
+        src = os.path.join(ROOT, kv["kernel_source"])
+        if hashlib.sha1(open(src, "rb").read()).hexdigest() != kv["kernel_source_sha1"]:
+            return None
+        return float(kv["dram_bytes_per_slot"]) * slots_per_launch
+    except (KeyError, OSError, ValueError):
+        return None
+
+
 # ---- integer schedule of the cache length (no scores involved) ---------------------------------
 def _after_prefill(N, w):
     if N < w.budget:
@@ -110,16 +131,6 @@ class ClockSampler:
         if sm:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
         return out
-
-
-def _decode_bytes(w, n):
-    """Algorithmic HBM bytes of one decode launch (one layer): per instance n K rows + n V rows +
-    score read/write (8 B per slot), plus q/k_new/v_new in and out."""
-    e = 2 if w.dtype == "bf16" else 4
-    inst = w.batch * w.kv_heads
-    per_slot = 2 * w.head_dim * e + 8
-    io = w.batch * (2 * w.q_heads + 2 * w.kv_heads) * w.head_dim * e
-    return inst * n * per_slot + io
 
 
 def run_ours(args):
@@ -235,8 +246,8 @@ def run_ours(args):
     bytes_all = w.layers * (slot_sum * w.kv_heads * per_slot + K * io)
     n_launch = w.layers * K
     achieved = bytes_all / (decode_ms * 1e-3) / 1e9
-    traffic = None   # ncu dram bytes per launch: see profiles/ (null once the kernel changed since)
-    roofline = dict(bound="hbm", kernel="decode_kernel", achieved=achieved, peak=peaks["hbm"], unit="GB/s",
+    traffic = _ncu_traffic(bytes_all / n_launch / per_slot if w.dtype == "bf16" else None)
+    roofline = dict(bound="hbm", kernel="decode_bf16_kernel" if w.dtype == "bf16" else "decode_kernel", achieved=achieved, peak=peaks["hbm"], unit="GB/s",
                     frac=achieved / peaks["hbm"], frac_of_nominal_8000=achieved / 8000.0, peak_source=peaks["source"],
                     traffic=traffic, bytes_per_launch=bytes_all / n_launch,
                     us_per_launch=decode_ms * 1e3 / n_launch)
