@@ -85,6 +85,20 @@ def _after_evict(n, n_old, w):
     return w.sink + m + w.window, m, True
 
 
+def max_over_ranks(value: float, dist, device) -> float:
+    """Slowest rank's time: every multi-GPU number is the max over ranks (replicas run independently)."""
+    if dist is None:
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank: float, world: int, ms: float) -> float:
+    """Aggregate throughput of `world` replicas that each processed units_per_rank in ms (max over ranks)."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
 class ClockSampler:
     """nvidia-smi sampling of SM clock and throttle reasons while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -235,10 +249,7 @@ def run_ours(args):
     launches = bz.launch_count() - l0
     ms = start.elapsed_time(end)
     assert bz.status() == 0
-    if dist:
-        tt = torch.tensor([ms], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms = tt.item()
+    ms = max_over_ranks(ms, dist, dev)
     decode_ms = sum(a.elapsed_time(b) for a, b in ev_pairs)
     # algorithmic bytes of all decode launches in the timed region (per layer the same lengths)
     per_slot = 2 * w.head_dim * esize + 8
@@ -271,13 +282,10 @@ def run_ours(args):
     e1.record(stream)
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1)
-    if dist:
-        tt = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = tt.item()
+    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
     h2d = w.layers * w.batch * (w.q_heads + 2 * w.kv_heads) * w.head_dim * esize
     d2h = w.layers * w.batch * w.q_heads * w.head_dim * esize
-    e2e = dict(value=world * w.batch * Ke / (e2e_ms * 1e-3), unit="tokens/s", steps=Ke,
+    e2e = dict(value=whole_job_rate(w.batch * Ke, world, e2e_ms), unit="tokens/s", steps=Ke,
                h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h)
     assert bz.status() == 0
 
@@ -308,7 +316,7 @@ def run_ours(args):
                      bytes=ev_bytes, at_step=t)
         assert bz.status() == 0
 
-    line = dict(metric="decode tokens/s (attention + BUZZ eviction)", value=world * w.batch * K / (ms * 1e-3),
+    line = dict(metric="decode tokens/s (attention + BUZZ eviction)", value=whole_job_rate(w.batch * K, world, ms),
                 unit="tokens/s", n_gpus=world, steps=K, warmup=W, ms_per_step=ms / K, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype=w.dtype, data="synthetic",
                 config=dict(workload=f"{w.name}: {w.layers} layers x {w.batch} seqs x {w.q_heads}/{w.kv_heads} heads, d={w.head_dim}, "
