@@ -8,8 +8,8 @@
 //   pass A  (attn_tc_kernel, query-tile stationary) flash-style attention: S in TMEM, one thread
 //           per row does the online softmax, P goes back to TMEM as bf16 and is the A operand of
 //           the P V MMA; the output accumulators live in TMEM and are rescaled lazily (only when a
-//           row maximum grows by more than 2^8). Two softmax warpgroups take alternate key tiles
-//           with an accumulator each and are merged at the end. Writes O and the row log2-sum-exp.
+//           row maximum grows by more than 2^8). Each row is shared by two threads (one per softmax
+//           warpgroup, half the columns each). Writes O and the row log2-sum-exp.
 //   pass B  (colsum_tc_kernel, key-tile stationary) S^T = K Q^T in TMEM with KEYS on the TMEM
 //           lanes, so one thread owns one key: it forms the exact probabilities 2^(S - lse) in
 //           fp32 and adds them up over the query rows in a fixed order (heads, then tiles, then
@@ -207,24 +207,27 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
 // =================================================================================================
 // Pass A: attention output and row log-sum-exp. grid (query tiles, query heads, sequences), 1 CTA/SM.
-// Two softmax warpgroups work on alternate key tiles, each with its own logits buffer and its own
-// output accumulator, so the exponentials of one tile overlap the MMAs of the other:
-//   TMEM columns: S0 [0,128)  S1 [128,256)  O0 [256,384)  O1 [384,512).
-// P (bf16 pairs) overwrites the first 64 columns of the S buffer it came from; the tensor core may
-// still be reading P as the A operand long after the MMA was issued, so the next logits for that
-// buffer are only issued once the P V product has been seen to complete (pv_done).
-// The two partial results (max, sum, output) of a row are merged in the epilogue.
+//   TMEM columns: S0 [0,128)  S1 [128,256)  P0 [256,320)  P1 [320,384) (bf16 pairs)  O [384,512).
+// The exponentials are the binding resource (16 per clock per SM, one warp per scheduler reaches a
+// quarter of that), so a query row is shared by TWO threads, one per softmax warpgroup: warpgroup
+// g owns columns [64g, 64g+64) of every logits tile. The two halves of a row exchange their
+// maxima through shared memory (one named barrier per tile), keep identical running maxima, and
+// add up their own part of the row sum; the halves are merged in the epilogue.
+// P has buffers of its own: the tensor core may still be reading P of tile j-1 as the A operand
+// while the logits of tile j+1 are being written, so it must not share columns with S.
 // =================================================================================================
 constexpr int kThreadsA = 320;            // TMA warp, MMA warp, 2 x 4 softmax warps
 struct SmemA {
   alignas(1024) unsigned char q[kTileBytes];
   alignas(1024) unsigned char k[3][kTileBytes];
   alignas(1024) unsigned char v[2][kTileBytes];
-  float xm[2][BT], xl[2][BT];             // per-row (max, sum) of each warpgroup, for the merge
-  uint64_t q_full, k_full[3], k_empty[3], v_full[2], v_empty[2], s_full[2], p_full[2], pv_done[2];
+  float xmax[2][2][BT];                   // [tile parity][warpgroup][row] half-row maxima
+  float xl[2][BT];                        // [warpgroup][row] half-row sums, for the epilogue
+  uint64_t q_full, k_full[3], k_empty[3], v_full[2], v_empty[2], s_full[2], p_full[2], o_done[2];
   uint32_t tmem_base;
 };
-constexpr uint32_t kColO = 256;
+constexpr uint32_t kColP = 256;
+constexpr uint32_t kColO = 384;
 constexpr float kRescaleThreshold = 8.0f;     // log2: rescale O only when a row max grows by > 2^8
 
 __global__ void __launch_bounds__(kThreadsA, 1)
@@ -248,7 +251,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     for (int s = 0; s < 3; ++s) { mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1); }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
-      mbar_init(&sm.s_full[s], 1); mbar_init(&sm.p_full[s], 128); mbar_init(&sm.pv_done[s], 1);
+      mbar_init(&sm.s_full[s], 1); mbar_init(&sm.p_full[s], 256); mbar_init(&sm.o_done[s], 1);
     }
     fence_barrier_init();
   }
@@ -296,139 +299,124 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       bool ok = mbar_wait(&sm.q_full, 0);
       if (!ok) tf.raise(14);
       ok = ok && issue_qk(0);
-      if (ok && nt > 1) ok = issue_qk(1);
       for (int j = 0; ok && j < nt; ++j) {
-        const int g = j & 1, u = j >> 1;
-        if (!mbar_wait(&sm.p_full[g], u & 1)) { tf.raise(15); break; }
-        if (!mbar_wait(&sm.v_full[g], u & 1)) { tf.raise(16); break; }
+        // S[(j+1)%2] was last read by the softmax of tile j-1, which has arrived on p_full(j-1)
+        if (j + 1 < nt && !issue_qk(j + 1)) break;     // next tile's logits overlap this tile's softmax
+        const int sb = j & 1, use = j >> 1;
+        if (!mbar_wait(&sm.p_full[sb], use & 1)) { tf.raise(15); break; }
+        if (!mbar_wait(&sm.v_full[sb], use & 1)) { tf.raise(16); break; }
         tc_fence_after();
-        const uint32_t va = smem_u32(sm.v[g]);
+        const uint32_t va = smem_u32(sm.v[sb]);
 #pragma unroll
-        for (int s = 0; s < BT / 16; ++s)              // O_g += P_j V_j, 16 keys per step
-          mma_ts(tmem + kColO + g * BT, tmem + g * BT + s * 8, mnmajor_desc(va, s), kIdescKM, (u > 0 || s > 0) ? 1u : 0u);
-        mma_commit(&sm.v_empty[g]);
-        mma_commit(&sm.pv_done[g]);
-        if (j + 2 < nt) {                              // S_g may be overwritten only once P_j has been consumed
-          if (!mbar_wait(&sm.pv_done[g], u & 1)) { tf.raise(21); break; }
-          if (!issue_qk(j + 2)) break;
-        }
+        for (int s = 0; s < BT / 16; ++s)              // O += P_j V_j, 16 keys per step
+          mma_ts(tmem + kColO, tmem + kColP + sb * 64 + s * 8, mnmajor_desc(va, s), kIdescKM, (j > 0 || s > 0) ? 1u : 0u);
+        mma_commit(&sm.v_empty[sb]);
+        mma_commit(&sm.o_done[sb]);
       }
     }
   } else {
-    // ---- softmax: one thread per query row and warpgroup; warpgroup g takes key tiles j = g, g+2, ... ----
+    // ---- softmax: thread (g, row) owns columns [64g, 64g+64) of the row's logits ----
     const int g = (warp - 2) >> 2;
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const int qpos = row0 + row;
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    const uint32_t colS = g * BT, colOg = kColO + g * BT;
     const float rs = scale_log2 * (logn ? __logf((float)(qpos + 1)) * kInvLn512 : 1.0f);
-    const int ntg = (nt - g + 1) >> 1;                 // tiles of this warpgroup
-    float m_used = -INFINITY, l = 0.f;
+    float m_used = -INFINITY, l = 0.f;                 // m_used is identical in both halves of a row
     bool ok = true;
-    for (int u = 0; u < ntg; ++u) {
-      const int j = 2 * u + g;
-      if (!mbar_wait(&sm.s_full[g], u & 1)) { tf.raise(17); ok = false; break; }
+    for (int j = 0; j < nt; ++j) {
+      const int sb = j & 1, use = j >> 1;
+      // (a thread that gave up on a wait keeps taking part in the named barriers, without waiting again)
+      if (ok && !mbar_wait(&sm.s_full[sb], use & 1)) { tf.raise(17); ok = false; }
       tc_fence_after();
-      // the raw logits of this row (rs > 0, so the row maximum can be taken before scaling)
-      float s[BT];
-#pragma unroll
-      for (int c0 = 0; c0 < BT; c0 += 32)
-        tmem_ld32(tmem + lane_base + colS + c0, *reinterpret_cast<uint32_t(*)[32]>(&s[c0]));
+      // the raw logits of this half row (rs > 0, so the maximum can be taken before scaling)
+      float s[64];
+      tmem_ld32(tmem + lane_base + sb * BT + g * 64, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+      tmem_ld32(tmem + lane_base + sb * BT + g * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
       tmem_wait_ld();
       if (j == nt - 1) {                               // the diagonal tile: causal mask
 #pragma unroll
-        for (int c = 0; c < BT; ++c)
-          if (j * BT + c > qpos) s[c] = -INFINITY;
+        for (int c = 0; c < 64; ++c)
+          if (j * BT + g * 64 + c > qpos) s[c] = -INFINITY;
       }
       float mx4[4] = {s[0], s[1], s[2], s[3]};
 #pragma unroll
-      for (int c = 4; c < BT; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], s[c]);
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * rs;
+      for (int c = 4; c < 64; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], s[c]);
+      const float mine = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      sm.xmax[sb][g][row] = mine;
+      asm volatile("bar.sync 2, 256;" ::: "memory");   // both halves of every row have published
+      const float mx = fmaxf(mine, sm.xmax[sb][g ^ 1][row]) * rs;
       const float m_new = fmaxf(m_used, mx);
-      if (u == 0) {
+      if (j == 0) {
         m_used = m_new;
       } else {
         const bool need = m_new > m_used + kRescaleThreshold;
-        if (__any_sync(0xffffffffu, need)) {            // rare after the first tiles
-          // O_g is idle here: these logits were only issued after the P V product of this
-          // warpgroup's previous tile had completed.
+        if (__any_sync(0xffffffffu, need)) {            // rare after the first tiles; same decision in both halves
           const float alpha = need ? exp2f(m_used - m_new) : 1.0f;
           if (need) m_used = m_new;
           l *= alpha;
+          if (ok && !mbar_wait(&sm.o_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; }   // P V of tile j-1 landed
+          tc_fence_after();
 #pragma unroll 1
-          for (int c0 = 0; c0 < D; c0 += 32) {
+          for (int c0 = g * 64; c0 < g * 64 + 64; c0 += 32) {   // this half rescales its 64 output columns
             uint32_t r[32];
-            tmem_ld32(tmem + lane_base + colOg + c0, r);
+            tmem_ld32(tmem + lane_base + kColO + c0, r);
             tmem_wait_ld();
 #pragma unroll
             for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
-            tmem_st32(tmem + lane_base + colOg + c0, r);
+            tmem_st32(tmem + lane_base + kColO + c0, r);
           }
           tmem_wait_st();
         }
       }
-      // P = 2^(S rs - m) as bf16 pairs over the first 64 columns of S_g (this row is in registers)
+      // P = 2^(S rs - m) as bf16 pairs into P[sb], once the P V product of tile j-2 has consumed it
+      if (ok && j >= 2 && !mbar_wait(&sm.o_done[sb], ((j >> 1) - 1) & 1)) { tf.raise(20); ok = false; }
       const float neg_m = -m_used;
       float l4[4] = {0.f, 0.f, 0.f, 0.f};
+      uint32_t pk[32];
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        uint32_t pk[32];
-#pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          const float p0 = exp2f(fmaf(s[half * 64 + 2 * c], rs, neg_m));
-          const float p1 = exp2f(fmaf(s[half * 64 + 2 * c + 1], rs, neg_m));
-          l4[c & 3] += p0 + p1;
-          const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
-          pk[c] = *reinterpret_cast<const uint32_t*>(&pp);
-        }
-        tmem_st32(tmem + lane_base + colS + half * 32, pk);
+      for (int c = 0; c < 32; ++c) {
+        const float p0 = exp2f(fmaf(s[2 * c], rs, neg_m));
+        const float p1 = exp2f(fmaf(s[2 * c + 1], rs, neg_m));
+        l4[c & 3] += p0 + p1;
+        const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
+        pk[c] = *reinterpret_cast<const uint32_t*>(&pp);
       }
+      tmem_st32(tmem + lane_base + kColP + sb * 64 + g * 32, pk);
       l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&sm.p_full[g]);
+      mbar_arrive(&sm.p_full[sb]);
     }
-    // ---- epilogue: merge the two warpgroups' partial results, O / l -> bf16, row log2-sum-exp ----
-    if (ok && ntg > 0 && !mbar_wait(&sm.pv_done[g], (ntg - 1) & 1)) { tf.raise(19); ok = false; }
+    // ---- epilogue: O / l -> bf16 (64 columns per half), row log2-sum-exp ----
+    if (ok && !mbar_wait(&sm.o_done[(nt - 1) & 1], ((nt - 1) >> 1) & 1)) { tf.raise(19); ok = false; }
     tc_fence_after();
-    sm.xm[g][row] = m_used;
     sm.xl[g][row] = l;
     asm volatile("bar.sync 2, 256;" ::: "memory");
-    const float m0 = sm.xm[0][row], m1 = sm.xm[1][row];
-    const float M = fmaxf(m0, m1);
-    const float f0 = exp2f(m0 - M);
-    const float f1 = (nt > 1) ? exp2f(m1 - M) : 0.f;   // warpgroup 1 has no tile when nt == 1
-    const float L = sm.xl[0][row] * f0 + sm.xl[1][row] * f1;
-    const float inv = 1.0f / L;
+    const float L = sm.xl[0][row] + sm.xl[1][row];
     if (ok) {
+      const float inv = 1.0f / L;
       __nv_bfloat16* orow = out + ((size_t)(tok0 + qpos) * Hq + h) * D;
 #pragma unroll 1
-      for (int c0 = g * 64; c0 < g * 64 + 64; c0 += 32) {   // warpgroup g writes output columns [64g, 64g+64)
-        uint32_t r0[32], r1[32];
-        tmem_ld32(tmem + lane_base + kColO + c0, r0);
-        if (nt > 1) tmem_ld32(tmem + lane_base + kColO + BT + c0, r1);
+      for (int c0 = g * 64; c0 < g * 64 + 64; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem + lane_base + kColO + c0, r);
         tmem_wait_ld();
         if (qpos < N) {
-          const float a0 = f0 * inv, a1 = f1 * inv;
 #pragma unroll
           for (int c = 0; c < 32; c += 8) {
-            float o[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              o[e] = __uint_as_float(r0[c + e]) * a0;
-              if (nt > 1) o[e] = fmaf(__uint_as_float(r1[c + e]), a1, o[e]);
-            }
             uint4 w;
-            __nv_bfloat162 t0 = __floats2bfloat162_rn(o[0], o[1]), t1 = __floats2bfloat162_rn(o[2], o[3]);
-            __nv_bfloat162 t2 = __floats2bfloat162_rn(o[4], o[5]), t3 = __floats2bfloat162_rn(o[6], o[7]);
+            __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(r[c]) * inv, __uint_as_float(r[c + 1]) * inv);
+            __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(r[c + 2]) * inv, __uint_as_float(r[c + 3]) * inv);
+            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(r[c + 4]) * inv, __uint_as_float(r[c + 5]) * inv);
+            __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(r[c + 6]) * inv, __uint_as_float(r[c + 7]) * inv);
             w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
             w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
             *reinterpret_cast<uint4*>(orow + c0 + c) = w;
           }
         }
       }
-      if (g == 0 && qpos < N) lse[(size_t)h * stride + tok0 + qpos] = M + log2f(L);
+      if (g == 0 && qpos < N) lse[(size_t)h * stride + tok0 + qpos] = m_used + log2f(L);
     }
   }
   tc_fence_before();
