@@ -9,7 +9,8 @@
 //           per row does the online softmax, P goes back to TMEM as bf16 and is the A operand of
 //           the P V MMA; the output accumulators live in TMEM and are rescaled lazily (only when a
 //           row maximum grows by more than 2^8). Each row is shared by two threads (one per softmax
-//           warpgroup, half the columns each). Writes O and the row log2-sum-exp.
+//           warpgroup, half the key columns and an accumulator each). Writes O and the row
+//           log2-sum-exp.
 //   pass B  (colsum_tc_kernel, key-tile stationary) S^T = K Q^T in TMEM with KEYS on the TMEM
 //           lanes, so one thread owns one key: it forms the exact probabilities 2^(S - lse) in
 //           fp32 and adds them up over the query rows in a fixed order (heads, then tiles, then
@@ -207,27 +208,29 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 
 // =================================================================================================
 // Pass A: attention output and row log-sum-exp. grid (query tiles, query heads, sequences), 1 CTA/SM.
-//   TMEM columns: S0 [0,128)  S1 [128,256)  P0 [256,320)  P1 [320,384) (bf16 pairs)  O [384,512).
-// The exponentials are the binding resource (16 per clock per SM, one warp per scheduler reaches a
-// quarter of that), so a query row is shared by TWO threads, one per softmax warpgroup: warpgroup
-// g owns columns [64g, 64g+64) of every logits tile. The two halves of a row exchange their
-// maxima through shared memory (one named barrier per tile), keep identical running maxima, and
-// add up their own part of the row sum; the halves are merged in the epilogue.
-// P has buffers of its own: the tensor core may still be reading P of tile j-1 as the A operand
-// while the logits of tile j+1 are being written, so it must not share columns with S.
+// The exponentials are the binding resource (16 per clock per SM; one warp per scheduler reaches a
+// quarter of that), so a query row is shared by TWO threads, one per softmax warpgroup: warpgroup g
+// owns key columns [64g, 64g+64) of every logits tile and runs a complete online softmax of its
+// own over them, with its own output accumulator (the P V product is split along the keys). The
+// warpgroups never synchronise inside the loop, so one can be taking maxima or waiting while the
+// other keeps the exponential unit busy; their (max, sum, output) are merged in the epilogue.
+//   TMEM columns: S0 [0,128)  S1 [128,256)  O_0 [256,384)  O_1 [384,512).
+// P_g (bf16 pairs, 32 columns) overwrites the start of the half row of S it was computed from.
+// The tensor core may still be reading P as the A operand long after the MMA was issued, so the
+// logits that reuse an S buffer are only issued once both P V products on it have been seen to
+// complete (pv_done).
 // =================================================================================================
 constexpr int kThreadsA = 320;            // TMA warp, MMA warp, 2 x 4 softmax warps
+constexpr int kStagesA = 3;
 struct SmemA {
   alignas(1024) unsigned char q[kTileBytes];
-  alignas(1024) unsigned char k[3][kTileBytes];
-  alignas(1024) unsigned char v[2][kTileBytes];
-  float xmax[2][2][BT];                   // [tile parity][warpgroup][row] half-row maxima
-  float xl[2][BT];                        // [warpgroup][row] half-row sums, for the epilogue
-  uint64_t q_full, k_full[3], k_empty[3], v_full[2], v_empty[2], s_full[2], p_full[2], o_done[2];
+  alignas(1024) unsigned char k[kStagesA][kTileBytes];
+  alignas(1024) unsigned char v[kStagesA][kTileBytes];
+  uint64_t q_full, k_full[kStagesA], k_empty[kStagesA], v_full[kStagesA], v_empty[kStagesA];
+  uint64_t s_full[2], p_full[2][2], pv_done[2];
   uint32_t tmem_base;
 };
-constexpr uint32_t kColP = 256;
-constexpr uint32_t kColO = 384;
+constexpr uint32_t kColO = 256;
 constexpr float kRescaleThreshold = 8.0f;     // log2: rescale O only when a row max grows by > 2^8
 
 __global__ void __launch_bounds__(kThreadsA, 1)
@@ -235,8 +238,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                const __grid_constant__ CUtensorMap map_v, const int32_t* __restrict__ cu,
                __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int32_t* status, int Hq, int Hkv,
                int stride, float scale_log2, int logn) {
-  extern __shared__ unsigned char smem_raw[];
-  SmemA& sm = *reinterpret_cast<SmemA*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  SmemA& sm = *reinterpret_cast<SmemA*>(smem_raw);
   const int b = blockIdx.z, h = blockIdx.y, kvh = h / (Hq / Hkv);
   const int tok0 = cu[b], N = cu[b + 1] - tok0;
   const int qt = gridDim.x - 1 - blockIdx.x;          // heaviest (last) query tiles first
@@ -245,13 +248,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nt = qt + 1;                              // key tiles 0..qt (causal)
   const TimeoutFlag tf{status, (b * Hq + h) * 4096 + qt};
+  if (smem_u32(smem_raw) & 1023u) {                   // the swizzled tiles need 1024-byte alignment
+    if (threadIdx.x == 0) buzz_set_status(status, BUZZ_ERR_INVALID, tf.inst, 30);
+    return;
+  }
 
   if (threadIdx.x == 0) {
     mbar_init(&sm.q_full, 1);
-    for (int s = 0; s < 3; ++s) { mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1); }
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < kStagesA; ++s) {
+      mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1);
       mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
-      mbar_init(&sm.s_full[s], 1); mbar_init(&sm.p_full[s], 256); mbar_init(&sm.o_done[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sm.s_full[s], 1); mbar_init(&sm.pv_done[s], 1);
+      mbar_init(&sm.p_full[s][0], 128); mbar_init(&sm.p_full[s][1], 128);
     }
     fence_barrier_init();
   }
@@ -271,13 +281,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_expect_tx(&sm.q_full, kTileBytes);
       load_tile(sm.q, &map_q, h * D, tok0 + row0, &sm.q_full);
       for (int j = 0; j < nt; ++j) {
-        const int ks = j % 3, ku = j / 3, vs = j & 1, vu = j >> 1;
-        if (ku > 0 && !mbar_wait(&sm.k_empty[ks], (ku - 1) & 1)) { tf.raise(11); break; }
-        mbar_expect_tx(&sm.k_full[ks], kTileBytes);
-        load_tile(sm.k[ks], &map_k, kvh * D, tok0 + j * BT, &sm.k_full[ks]);
-        if (vu > 0 && !mbar_wait(&sm.v_empty[vs], (vu - 1) & 1)) { tf.raise(12); break; }
-        mbar_expect_tx(&sm.v_full[vs], kTileBytes);
-        load_tile(sm.v[vs], &map_v, kvh * D, tok0 + j * BT, &sm.v_full[vs]);
+        const int st = j % kStagesA, use = j / kStagesA;
+        if (use > 0 && !mbar_wait(&sm.k_empty[st], (use - 1) & 1)) { tf.raise(11); break; }
+        mbar_expect_tx(&sm.k_full[st], kTileBytes);
+        load_tile(sm.k[st], &map_k, kvh * D, tok0 + j * BT, &sm.k_full[st]);
+        if (use > 0 && !mbar_wait(&sm.v_empty[st], (use - 1) & 1)) { tf.raise(12); break; }
+        mbar_expect_tx(&sm.v_full[st], kTileBytes);
+        load_tile(sm.v[st], &map_v, kvh * D, tok0 + j * BT, &sm.v_full[st]);
       }
     }
   } else if (warp == 1) {
@@ -285,54 +295,63 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (elect_one()) {
       const uint32_t qa = smem_u32(sm.q);
       auto issue_qk = [&](int j) -> bool {             // S[j%2] = Q K_j^T
-        const int ks = j % 3;
-        if (!mbar_wait(&sm.k_full[ks], (j / 3) & 1)) { tf.raise(13); return false; }
+        const int st = j % kStagesA;
+        if (!mbar_wait(&sm.k_full[st], (j / kStagesA) & 1)) { tf.raise(13); return false; }
         tc_fence_after();
-        const uint32_t ka = smem_u32(sm.k[ks]);
+        const uint32_t ka = smem_u32(sm.k[st]);
 #pragma unroll
         for (int s = 0; s < D / 16; ++s)
           mma_ss(tmem + (j & 1) * BT, kmajor_desc(qa, s), kmajor_desc(ka, s), kIdescKK, s > 0);
         mma_commit(&sm.s_full[j & 1]);
-        mma_commit(&sm.k_empty[ks]);
+        mma_commit(&sm.k_empty[st]);
         return true;
       };
       bool ok = mbar_wait(&sm.q_full, 0);
       if (!ok) tf.raise(14);
       ok = ok && issue_qk(0);
       for (int j = 0; ok && j < nt; ++j) {
-        // S[(j+1)%2] was last read by the softmax of tile j-1, which has arrived on p_full(j-1)
-        if (j + 1 < nt && !issue_qk(j + 1)) break;     // next tile's logits overlap this tile's softmax
-        const int sb = j & 1, use = j >> 1;
-        if (!mbar_wait(&sm.p_full[sb], use & 1)) { tf.raise(15); break; }
-        if (!mbar_wait(&sm.v_full[sb], use & 1)) { tf.raise(16); break; }
-        tc_fence_after();
-        const uint32_t va = smem_u32(sm.v[sb]);
+        if (j + 1 < nt) {
+          // S[(j+1)%2] still holds P of tile j-1: both of its P V products must have completed
+          if (j >= 1 && !mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(21); break; }
+          if (!issue_qk(j + 1)) break;                 // next tile's logits overlap this tile's softmax
+        }
+        const int sb = j & 1, st = j % kStagesA;
+        bool fine = true;
+        for (int g = 0; g < 2 && fine; ++g) {          // O_g += P_g V[64g .. 64g+63], 16 keys per step
+          if (!mbar_wait(&sm.p_full[sb][g], (j >> 1) & 1)) { tf.raise(15); fine = false; break; }
+          if (g == 0 && !mbar_wait(&sm.v_full[st], (j / kStagesA) & 1)) { tf.raise(16); fine = false; break; }
+          tc_fence_after();
+          const uint32_t va = smem_u32(sm.v[st]);
 #pragma unroll
-        for (int s = 0; s < BT / 16; ++s)              // O += P_j V_j, 16 keys per step
-          mma_ts(tmem + kColO, tmem + kColP + sb * 64 + s * 8, mnmajor_desc(va, s), kIdescKM, (j > 0 || s > 0) ? 1u : 0u);
-        mma_commit(&sm.v_empty[sb]);
-        mma_commit(&sm.o_done[sb]);
+          for (int s = 0; s < 4; ++s)
+            mma_ts(tmem + kColO + g * BT, tmem + sb * BT + g * 64 + s * 8, mnmajor_desc(va, g * 4 + s), kIdescKM,
+                   (j > 0 || s > 0) ? 1u : 0u);
+        }
+        if (!fine) break;
+        mma_commit(&sm.v_empty[st]);
+        mma_commit(&sm.pv_done[sb]);
       }
     }
   } else {
-    // ---- softmax: thread (g, row) owns columns [64g, 64g+64) of the row's logits ----
+    // ---- softmax: thread (g, row) runs an online softmax over key columns [64g, 64g+64) of every tile ----
     const int g = (warp - 2) >> 2;
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const int qpos = row0 + row;
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const uint32_t colOg = kColO + g * BT;
     const float rs = scale_log2 * (logn ? __logf((float)(qpos + 1)) * kInvLn512 : 1.0f);
-    float m_used = -INFINITY, l = 0.f;                 // m_used is identical in both halves of a row
+    float m_used = -INFINITY, l = 0.f;
     bool ok = true;
     for (int j = 0; j < nt; ++j) {
-      const int sb = j & 1, use = j >> 1;
-      // (a thread that gave up on a wait keeps taking part in the named barriers, without waiting again)
-      if (ok && !mbar_wait(&sm.s_full[sb], use & 1)) { tf.raise(17); ok = false; }
+      const int sb = j & 1;
+      const uint32_t colS = sb * BT + g * 64;
+      if (!mbar_wait(&sm.s_full[sb], (j >> 1) & 1)) { tf.raise(17); ok = false; break; }
       tc_fence_after();
       // the raw logits of this half row (rs > 0, so the maximum can be taken before scaling)
       float s[64];
-      tmem_ld32(tmem + lane_base + sb * BT + g * 64, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-      tmem_ld32(tmem + lane_base + sb * BT + g * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+      tmem_ld32(tmem + lane_base + colS, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+      tmem_ld32(tmem + lane_base + colS + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
       tmem_wait_ld();
       if (j == nt - 1) {                               // the diagonal tile: causal mask
 #pragma unroll
@@ -342,36 +361,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       float mx4[4] = {s[0], s[1], s[2], s[3]};
 #pragma unroll
       for (int c = 4; c < 64; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], s[c]);
-      const float mine = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      sm.xmax[sb][g][row] = mine;
-      asm volatile("bar.sync 2, 256;" ::: "memory");   // both halves of every row have published
-      const float mx = fmaxf(mine, sm.xmax[sb][g ^ 1][row]) * rs;
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * rs;   // -inf if the half row is masked out
       const float m_new = fmaxf(m_used, mx);
       if (j == 0) {
         m_used = m_new;
       } else {
         const bool need = m_new > m_used + kRescaleThreshold;
-        if (__any_sync(0xffffffffu, need)) {            // rare after the first tiles; same decision in both halves
-          const float alpha = need ? exp2f(m_used - m_new) : 1.0f;
+        if (__any_sync(0xffffffffu, need)) {
+          const float alpha = need ? exp2f(m_used - m_new) : 1.0f;     // 0 when nothing was unmasked so far
           if (need) m_used = m_new;
           l *= alpha;
-          if (ok && !mbar_wait(&sm.o_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; }   // P V of tile j-1 landed
+          if (!mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
           tc_fence_after();
 #pragma unroll 1
-          for (int c0 = g * 64; c0 < g * 64 + 64; c0 += 32) {   // this half rescales its 64 output columns
+          for (int c0 = 0; c0 < D; c0 += 32) {
             uint32_t r[32];
-            tmem_ld32(tmem + lane_base + kColO + c0, r);
+            tmem_ld32(tmem + lane_base + colOg + c0, r);
             tmem_wait_ld();
 #pragma unroll
             for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
-            tmem_st32(tmem + lane_base + kColO + c0, r);
+            tmem_st32(tmem + lane_base + colOg + c0, r);
           }
           tmem_wait_st();
         }
       }
-      // P = 2^(S rs - m) as bf16 pairs into P[sb], once the P V product of tile j-2 has consumed it
-      if (ok && j >= 2 && !mbar_wait(&sm.o_done[sb], ((j >> 1) - 1) & 1)) { tf.raise(20); ok = false; }
-      const float neg_m = -m_used;
+      // P_g = 2^(S rs - m) as bf16 pairs over the first 32 columns of this half row (which is in registers)
+      const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
       float l4[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pk[32];
 #pragma unroll
@@ -382,41 +397,51 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
         pk[c] = *reinterpret_cast<const uint32_t*>(&pp);
       }
-      tmem_st32(tmem + lane_base + kColP + sb * 64 + g * 32, pk);
+      tmem_st32(tmem + lane_base + colS, pk);
       l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&sm.p_full[sb]);
+      mbar_arrive(&sm.p_full[sb][g]);
     }
-    // ---- epilogue: O / l -> bf16 (64 columns per half), row log2-sum-exp ----
-    if (ok && !mbar_wait(&sm.o_done[(nt - 1) & 1], ((nt - 1) >> 1) & 1)) { tf.raise(19); ok = false; }
+    // ---- epilogue: merge the two halves of the row, O / l -> bf16, row log2-sum-exp ----
+    if (ok && !mbar_wait(&sm.pv_done[(nt - 1) & 1], ((nt - 1) >> 1) & 1)) { tf.raise(19); ok = false; }
     tc_fence_after();
-    sm.xl[g][row] = l;
+    // the K ring is idle now (its last use completed before that P V product): exchange (max, sum) there
+    float* xm = reinterpret_cast<float*>(sm.k[0]);    // [2][BT]
+    float* xl = xm + 2 * BT;                           // [2][BT]
+    xm[g * BT + row] = m_used;
+    xl[g * BT + row] = l;
     asm volatile("bar.sync 2, 256;" ::: "memory");
-    const float L = sm.xl[0][row] + sm.xl[1][row];
+    const float m0 = xm[row], m1 = xm[BT + row];
+    const float M = fmaxf(m0, m1);                     // finite: key 0 is never masked for any row
+    const float f0 = (m0 == -INFINITY) ? 0.f : exp2f(m0 - M);
+    const float f1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - M);
+    const float L = xl[row] * f0 + xl[BT + row] * f1;
     if (ok) {
-      const float inv = 1.0f / L;
+      const float a0 = f0 / L, a1 = f1 / L;
       __nv_bfloat16* orow = out + ((size_t)(tok0 + qpos) * Hq + h) * D;
 #pragma unroll 1
-      for (int c0 = g * 64; c0 < g * 64 + 64; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(tmem + lane_base + kColO + c0, r);
+      for (int c0 = g * 64; c0 < g * 64 + 64; c0 += 32) {   // warpgroup g writes output columns [64g, 64g+64)
+        uint32_t r0[32], r1[32];
+        tmem_ld32(tmem + lane_base + kColO + c0, r0);
+        tmem_ld32(tmem + lane_base + kColO + BT + c0, r1);
         tmem_wait_ld();
         if (qpos < N) {
 #pragma unroll
           for (int c = 0; c < 32; c += 8) {
+            float o[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) o[e] = fmaf(__uint_as_float(r1[c + e]), a1, __uint_as_float(r0[c + e]) * a0);
             uint4 w;
-            __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(r[c]) * inv, __uint_as_float(r[c + 1]) * inv);
-            __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(r[c + 2]) * inv, __uint_as_float(r[c + 3]) * inv);
-            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(r[c + 4]) * inv, __uint_as_float(r[c + 5]) * inv);
-            __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(r[c + 6]) * inv, __uint_as_float(r[c + 7]) * inv);
+            __nv_bfloat162 t0 = __floats2bfloat162_rn(o[0], o[1]), t1 = __floats2bfloat162_rn(o[2], o[3]);
+            __nv_bfloat162 t2 = __floats2bfloat162_rn(o[4], o[5]), t3 = __floats2bfloat162_rn(o[6], o[7]);
             w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
             w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
             *reinterpret_cast<uint4*>(orow + c0 + c) = w;
           }
         }
       }
-      if (g == 0 && qpos < N) lse[(size_t)h * stride + tok0 + qpos] = m_used + log2f(L);
+      if (g == 0 && qpos < N) lse[(size_t)h * stride + tok0 + qpos] = M + log2f(L);
     }
   }
   tc_fence_before();
@@ -467,7 +492,7 @@ cudaError_t buzz_launch_prefill_tc(buzz_ctx* c, const void* q, const void* k, co
   if (!make_map(&mq, q, total_tokens, c->sh.q_heads) || !make_map(&mk, k, total_tokens, c->sh.kv_heads) ||
       !make_map(&mv, v, total_tokens, c->sh.kv_heads))
     return cudaErrorInvalidValue;
-  const size_t smemA = sizeof(SmemA) + 1024, smemB = sizeof(SmemB) + 1024;
+  const size_t smemA = sizeof(SmemA), smemB = sizeof(SmemB) + 1024;
   static bool attr_done = false;
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smemA);
