@@ -59,19 +59,19 @@ __device__ __forceinline__ void load_tile(void* dst, const CUtensorMap* map, int
 
 // One key's 128 logits against one query tile -> exact probabilities added into four interleaved
 // accumulators (column c -> acc[c % 4]), so the summation order is fixed and the adds pipeline.
-template <bool LOGN>
-__device__ __forceinline__ void colsum_tile(const uint32_t (&r)[BT], const float* __restrict__ rs,
+template <bool LOGN, int NC>
+__device__ __forceinline__ void colsum_tile(const uint32_t (&r)[NC], const float* __restrict__ rs,
                                             const float* __restrict__ lse, float scale_log2, bool diag,
                                             bool tail, int q0, int kpos, int N, float (&acc)[4]) {
   if (!diag && !tail) {
 #pragma unroll
-    for (int c = 0; c < BT; ++c) {
+    for (int c = 0; c < NC; ++c) {
       const float sc = LOGN ? rs[c] : scale_log2;
       acc[c & 3] += exp2f(fmaf(__uint_as_float(r[c]), sc, -lse[c]));
     }
   } else {
 #pragma unroll
-    for (int c = 0; c < BT; ++c) {
+    for (int c = 0; c < NC; ++c) {
       const float sc = LOGN ? rs[c] : scale_log2;
       const float p = exp2f(fmaf(__uint_as_float(r[c]), sc, -lse[c]));
       const int qpos = q0 + c;
@@ -81,18 +81,22 @@ __device__ __forceinline__ void colsum_tile(const uint32_t (&r)[BT], const float
 }
 
 // =================================================================================================
-// Pass B: column sums. grid (key tiles, kv heads, sequences), 2 CTAs per SM.
+// Pass B: column sums. grid (key tiles, kv heads, sequences), 2 CTAs per SM. A key (TMEM lane) is
+// shared by two threads, one per compute warpgroup: warpgroup g sums query columns [64g, 64g+64)
+// of every tile, and the two partial sums are added in a fixed order at the end.
 // =================================================================================================
 struct SmemB {
   alignas(1024) unsigned char k[kTileBytes];
   alignas(1024) unsigned char q[2][kTileBytes];
   float lse[2][BT];
   float rs[2][BT];
+  float part[BT];                          // warpgroup 1's partial column sums
   uint64_t k_full, q_full[2], q_empty[2], s_full[2], s_empty[2];
   uint32_t tmem_base;
 };
 
-__global__ void __launch_bounds__(kThreads, 2)
+constexpr int kThreadsB = 320;            // TMA warp, MMA warp, 2 x 4 compute warps
+__global__ void __launch_bounds__(kThreadsB, 2)
 colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const int32_t* __restrict__ cu, const float* __restrict__ lse, float* __restrict__ pscore,
                  int32_t* status, int Hq, int Hkv, int stride, float scale_log2, int logn) {
@@ -114,7 +118,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       mbar_init(&sm.q_full[s], 1);
       mbar_init(&sm.q_empty[s], 1);
       mbar_init(&sm.s_full[s], 1);
-      mbar_init(&sm.s_empty[s], 128);
+      mbar_init(&sm.s_empty[s], 256);
     }
     fence_barrier_init();
   }
@@ -161,42 +165,46 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       }
     }
   } else {
-    // ---- one thread per key: exact probabilities, summed down the column ----
+    // ---- thread (g, key): exact probabilities of query columns [64g, 64g+64), summed down the column ----
+    const int g = (warp - 2) >> 2;
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;              // TMEM lane = key within the tile
-    const int t = (warp - 2) * 32 + lane;             // 0..127 among the compute threads
+    const int t = (warp - 2) * 32 + lane;             // 0..255 among the compute threads
     const int kpos = key0 + row;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};           // column c adds into acc[c % 4]: a fixed order
+    bool ok = true;
     for (int it = 0; it < iters; ++it) {
       const int st = it & 1, use = it >> 1;
-      const int g = it / nq, qt = kt + it % nq;
+      const int gq = it / nq, qt = kt + it % nq;
       const int q0 = qt * BT;
-      const int h = kvh * G + g;
+      const int h = kvh * G + gq;
       // stage this tile's row statistics; the named barrier below publishes them
-      {
+      if (t < BT) {
         const int qpos = q0 + t;
         sm.lse[st][t] = (qpos < N) ? lse[(size_t)h * stride + tok0 + qpos] : 0.f;
         sm.rs[st][t] = scale_log2 * (logn ? __logf((float)(qpos + 1)) * kInvLn512 : 1.0f);
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (!mbar_wait(&sm.s_full[st], use & 1)) { tf.raise(5); break; }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      // (a thread that gave up on a wait keeps taking part in the named barriers, without waiting again)
+      if (ok && !mbar_wait(&sm.s_full[st], use & 1)) { tf.raise(5); ok = false; }
       tc_fence_after();
       const bool diag = (qt == kt), tail = (q0 + BT > N);
-      // the whole row of S^T first (four loads in flight), then 128 independent exponentials
-      uint32_t r[BT];
-#pragma unroll
-      for (int c0 = 0; c0 < BT; c0 += 32)
-        tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + st * BT + c0, *reinterpret_cast<uint32_t(*)[32]>(&r[c0]));
+      // this thread's 64 logits first (two loads in flight), then 64 independent exponentials
+      uint32_t r[64];
+      tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + st * BT + g * 64, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+      tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + st * BT + g * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
       tmem_wait_ld();
       tc_fence_before();
-      mbar_arrive(&sm.s_empty[st]);                    // S^T[st] may be overwritten from here on
-      if (logn) colsum_tile<true>(r, sm.rs[st], sm.lse[st], scale_log2, diag, tail, q0, kpos, N, acc);
-      else colsum_tile<false>(r, sm.rs[st], sm.lse[st], scale_log2, diag, tail, q0, kpos, N, acc);
-
+      mbar_arrive(&sm.s_empty[st]);                    // S^T[st] may be overwritten once all 256 have arrived
+      if (logn) colsum_tile<true, 64>(r, sm.rs[st] + g * 64, sm.lse[st] + g * 64, scale_log2, diag, tail, q0 + g * 64, kpos, N, acc);
+      else colsum_tile<false, 64>(r, sm.rs[st] + g * 64, sm.lse[st] + g * 64, scale_log2, diag, tail, q0 + g * 64, kpos, N, acc);
       // lse[st]/rs[st] are restaged two iterations from now; the named barrier of the next
       // iteration, which every thread reaches only after these reads, orders that.
     }
-    if (kpos < N) pscore[(size_t)kvh * stride + tok0 + kpos] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    const float mine = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    if (g == 1) sm.part[row] = mine;
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (g == 0 && ok && kpos < N) pscore[(size_t)kvh * stride + tok0 + kpos] = mine + sm.part[row];
   }
   tc_fence_before();
   __syncthreads();
@@ -231,7 +239,8 @@ struct SmemA {
   uint32_t tmem_base;
 };
 constexpr uint32_t kColO = 256;
-constexpr float kRescaleThreshold = 8.0f;     // log2: rescale O only when a row max grows by > 2^8
+constexpr float kRescaleThreshold = 20.0f;    // log2: rescale O only when a row max grows by > 2^20
+                                              // (P, the row sums and O stay far inside the fp32/bf16 exponent range)
 
 __global__ void __launch_bounds__(kThreadsA, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -509,7 +518,7 @@ cudaError_t buzz_launch_prefill_tc(buzz_ctx* c, const void* q, const void* k, co
       c->sh.max_prompt_tokens, scale_log2, logn);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  colsum_tc_kernel<<<dim3(tiles, c->sh.kv_heads, batch), kThreads, smemB, stream>>>(
+  colsum_tc_kernel<<<dim3(tiles, c->sh.kv_heads, batch), kThreadsB, smemB, stream>>>(
       mq, mk, cu, c->lse, c->pscore, c->st.status, c->sh.q_heads, c->sh.kv_heads, c->sh.max_prompt_tokens,
       scale_log2, logn);
   *launches += 2;
