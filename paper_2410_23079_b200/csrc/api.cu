@@ -52,7 +52,7 @@ Layout make_layout(const buzz_shape& s, int budget) {
   L.status = off; off = align_up(off + 4 * sizeof(int32_t));
   L.state_bytes = off;
   off = 0;
-  L.lse = off; off = align_up(off + (size_t)s.q_heads * buzz_lse_stride(s) * sizeof(float));
+  L.lse = off; off = align_up(off + (size_t)s.q_heads * s.max_prompt_tokens * sizeof(float));
   L.pscore = off; off = align_up(off + (size_t)s.kv_heads * s.max_prompt_tokens * sizeof(float));
   L.stage_q = align_up((size_t)s.max_batch * s.q_heads * s.head_dim * e);
   L.stage_kv = align_up((size_t)s.max_batch * s.kv_heads * s.head_dim * e);

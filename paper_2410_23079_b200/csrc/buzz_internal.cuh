@@ -46,10 +46,6 @@ struct buzz_ctx {
   long long launches;
 };
 
-// Floats per query head in the row-statistics scratch: the packed prompt, padded so that every
-// sequence starts 16-byte aligned and owns a whole number of 128-row tiles.
-inline int buzz_lse_stride(const buzz_shape& sh) { return ((sh.max_prompt_tokens + 3) & ~3) + 128 * sh.max_batch + 4; }
-
 __host__ __device__ inline size_t buzz_inst(const buzz_shape& sh, int layer, int seq, int head) {
   return ((size_t)layer * sh.max_batch + seq) * sh.kv_heads + head;
 }

@@ -51,10 +51,6 @@ __device__ __forceinline__ uint64_t mnmajor_desc(uint32_t tile_saddr, int ks) {
   return smem_desc_sw128(tile_saddr + ks * 16 * 128, kBlockBytes, 1024);
 }
 
-// Row statistics of the tensor-core path are kept per (head, sequence) at a 16-byte aligned offset with
-// room for a whole number of 128-row tiles, so a tile's 128 values can be read four at a time.
-__host__ __device__ __forceinline__ int lse_offset(int tok0, int seq) { return ((tok0 + 3) & ~3) + BT * seq; }
-
 // One [128 x 128] bf16 tile = two TMA boxes of 64 columns.
 __device__ __forceinline__ void load_tile(void* dst, const CUtensorMap* map, int col0, int row0, uint64_t* bar) {
   tma_load_2d(dst, map, col0, row0, bar);
@@ -67,26 +63,19 @@ template <bool LOGN, int NC>
 __device__ __forceinline__ void colsum_tile(const uint32_t (&r)[NC], const float* __restrict__ rs,
                                             const float* __restrict__ lse, float scale_log2, bool diag,
                                             bool tail, int q0, int kpos, int N, float (&acc)[4]) {
-  // lse (and rs) are 16-byte aligned and read four at a time: the same addresses in every lane
-  const float4* lse4 = reinterpret_cast<const float4*>(lse);
-  const float4* rs4 = reinterpret_cast<const float4*>(rs);
-  const bool masked = diag || tail;
+  if (!diag && !tail) {
 #pragma unroll
-  for (int c4 = 0; c4 < NC / 4; ++c4) {
-    const float4 lv = lse4[c4];
-    float4 sv = make_float4(scale_log2, scale_log2, scale_log2, scale_log2);
-    if (LOGN) sv = rs4[c4];
-    const float lq[4] = {lv.x, lv.y, lv.z, lv.w};
-    const float sq[4] = {sv.x, sv.y, sv.z, sv.w};
+    for (int c = 0; c < NC; ++c) {
+      const float sc = LOGN ? rs[c] : scale_log2;
+      acc[c & 3] += exp2f(fmaf(__uint_as_float(r[c]), sc, -lse[c]));
+    }
+  } else {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int c = c4 * 4 + e;
-      float p = exp2f(fmaf(__uint_as_float(r[c]), sq[e], -lq[e]));
-      if (masked) {
-        const int qpos = q0 + c;
-        p = (qpos >= kpos && qpos < N) ? p : 0.f;
-      }
-      acc[e] += p;
+    for (int c = 0; c < NC; ++c) {
+      const float sc = LOGN ? rs[c] : scale_log2;
+      const float p = exp2f(fmaf(__uint_as_float(r[c]), sc, -lse[c]));
+      const int qpos = q0 + c;
+      acc[c & 3] += (qpos >= kpos && qpos < N) ? p : 0.f;
     }
   }
 }
@@ -110,7 +99,7 @@ constexpr int kThreadsB = 320;            // TMA warp, MMA warp, 2 x 4 compute w
 __global__ void __launch_bounds__(kThreadsB, 2)
 colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const int32_t* __restrict__ cu, const float* __restrict__ lse, float* __restrict__ pscore,
-                 int32_t* status, int Hq, int Hkv, int stride, int lstride, float scale_log2, int logn) {
+                 int32_t* status, int Hq, int Hkv, int stride, float scale_log2, int logn) {
   extern __shared__ unsigned char smem_raw[];
   SmemB& sm = *reinterpret_cast<SmemB*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int b = blockIdx.z, kvh = blockIdx.y, G = Hq / Hkv;
@@ -182,7 +171,6 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int row = quarter * 32 + lane;              // TMEM lane = key within the tile
     const int t = (warp - 2) * 32 + lane;             // 0..255 among the compute threads
     const int kpos = key0 + row;
-    const float* lse_al = lse + lse_offset(tok0, b);   // 16-byte aligned, padded per sequence
     float acc[4] = {0.f, 0.f, 0.f, 0.f};           // column c adds into acc[c % 4]: a fixed order
     bool ok = true;
     for (int it = 0; it < iters; ++it) {
@@ -190,15 +178,13 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       const int gq = it / nq, qt = kt + it % nq;
       const int q0 = qt * BT;
       const int h = kvh * G + gq;
-      if (logn) {
-        // per-row logit scales differ: stage them (and lse) in shared memory; the named barrier publishes them
-        if (t < BT) {
-          const int qpos = q0 + t;
-          sm.lse[st][t] = (qpos < N) ? lse_al[(size_t)h * lstride + qpos] : 0.f;
-          sm.rs[st][t] = scale_log2 * __logf((float)(qpos + 1)) * kInvLn512;
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
+      // stage this tile's row statistics; the named barrier below publishes them
+      if (t < BT) {
+        const int qpos = q0 + t;
+        sm.lse[st][t] = (qpos < N) ? lse[(size_t)h * stride + tok0 + qpos] : 0.f;
+        sm.rs[st][t] = scale_log2 * (logn ? __logf((float)(qpos + 1)) * kInvLn512 : 1.0f);
       }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
       // (a thread that gave up on a wait keeps taking part in the named barriers, without waiting again)
       if (ok && !mbar_wait(&sm.s_full[st], use & 1)) { tf.raise(5); ok = false; }
       tc_fence_after();
@@ -210,13 +196,8 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(&sm.s_empty[st]);                    // S^T[st] may be overwritten once all 256 have arrived
-      if (logn) {
-        colsum_tile<true, 64>(r, sm.rs[st] + g * 64, sm.lse[st] + g * 64, scale_log2, diag, tail, q0 + g * 64, kpos, N, acc);
-      } else {
-        // the row statistics straight from global memory (L1-resident, one address per warp-wide load);
-        // entries beyond the sequence are never used unmasked
-        colsum_tile<false, 64>(r, nullptr, lse_al + (size_t)h * lstride + q0 + g * 64, scale_log2, diag, tail, q0 + g * 64, kpos, N, acc);
-      }
+      if (logn) colsum_tile<true, 64>(r, sm.rs[st] + g * 64, sm.lse[st] + g * 64, scale_log2, diag, tail, q0 + g * 64, kpos, N, acc);
+      else colsum_tile<false, 64>(r, sm.rs[st] + g * 64, sm.lse[st] + g * 64, scale_log2, diag, tail, q0 + g * 64, kpos, N, acc);
       // lse[st]/rs[st] are restaged two iterations from now; the named barrier of the next
       // iteration, which every thread reaches only after these reads, orders that.
     }
@@ -265,7 +246,7 @@ __global__ void __launch_bounds__(kThreadsA, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const int32_t* __restrict__ cu,
                __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int32_t* status, int Hq, int Hkv,
-               int lstride, float scale_log2, int logn) {
+               int stride, float scale_log2, int logn) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   SmemA& sm = *reinterpret_cast<SmemA*>(smem_raw);
   const int b = blockIdx.z, h = blockIdx.y, kvh = h / (Hq / Hkv);
@@ -469,7 +450,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           }
         }
       }
-      if (g == 0 && qpos < N) lse[(size_t)h * lstride + lse_offset(tok0, b) + qpos] = M + log2f(L);
+      if (g == 0 && qpos < N) lse[(size_t)h * stride + tok0 + qpos] = M + log2f(L);
     }
   }
   tc_fence_before();
@@ -534,12 +515,12 @@ cudaError_t buzz_launch_prefill_tc(buzz_ctx* c, const void* q, const void* k, co
   const int logn = (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0;
   attn_tc_kernel<<<dim3(tiles, c->sh.q_heads, batch), kThreadsA, smemA, stream>>>(
       mq, mk, mv, cu, (__nv_bfloat16*)out, c->lse, c->st.status, c->sh.q_heads, c->sh.kv_heads,
-      buzz_lse_stride(c->sh), scale_log2, logn);
+      c->sh.max_prompt_tokens, scale_log2, logn);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   colsum_tc_kernel<<<dim3(tiles, c->sh.kv_heads, batch), kThreadsB, smemB, stream>>>(
       mq, mk, cu, c->lse, c->pscore, c->st.status, c->sh.q_heads, c->sh.kv_heads, c->sh.max_prompt_tokens,
-      buzz_lse_stride(c->sh), scale_log2, logn);
+      scale_log2, logn);
   *launches += 2;
   return cudaGetLastError();
 }
