@@ -113,6 +113,7 @@ int buzz_create(buzz_t* out, int sink, int window, int segment, int hitters, int
   c->batch = static_cast<int*>(calloc(shape->layers, sizeof(int)));
   c->decode_cluster = 0;
   c->launches = 0;
+  c->last_kind = 0; c->last_layer = -1; c->last_stream = nullptr;
   if (!c->batch) { delete c; return BUZZ_ERR_INVALID; }
   if (cudaMemset(state_dev, 0, L.state_bytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
     free(c->batch);
@@ -238,6 +239,7 @@ int buzz_import_state(buzz_t c, int layer, int seq, int kv_head, int32_t n, int3
   if (cudaMemcpy(c->st.n_old + inst, &cnt[1], 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
   if (cudaMemcpy(c->st.total + inst, &cnt[2], 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
   if (c->batch[layer] < seq + 1) c->batch[layer] = seq + 1;
+  c->last_kind = 2;
   return BUZZ_OK;
 }
 

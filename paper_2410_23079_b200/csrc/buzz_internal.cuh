@@ -44,6 +44,9 @@ struct buzz_ctx {
   int* batch;         // active sequences per layer (host array)
   int decode_cluster; // 0 = choose automatically
   long long launches;
+  // what the library launched last through this object (0 nothing, 1 a bf16 decode step, 2 anything else)
+  int last_kind, last_layer;
+  void* last_stream;
 };
 
 __host__ __device__ inline size_t buzz_inst(const buzz_shape& sh, int layer, int seq, int head) {

@@ -332,7 +332,7 @@ cudaError_t launch_g(buzz_ctx* c, int layer, const void* q, const void* k_new, c
 }  // namespace
 
 cudaError_t buzz_launch_decode_bf16(buzz_ctx* c, int layer, const void* q, const void* k_new,
-                                    const void* v_new, void* out, int cluster_size, cudaStream_t stream);
+                                    const void* v_new, void* out, int cluster_size, int early, cudaStream_t stream);
 
 cudaError_t buzz_launch_decode(buzz_ctx* c, int layer, const void* q, const void* k_new,
                                const void* v_new, void* out, cudaStream_t stream) {
@@ -350,10 +350,15 @@ cudaError_t buzz_launch_decode(buzz_ctx* c, int layer, const void* q, const void
   while (cs < kMaxCluster && (size_t)c->group * ((c->pol.budget + cs - 1) / cs) * sizeof(float) > 96 * 1024) cs *= 2;
   cudaError_t e;
   if (c->sh.dtype == BUZZ_BF16) {
-    e = buzz_launch_decode_bf16(c, layer, q, k_new, v_new, out, cs, stream);   // tensor-core kernel
+    // the kernel may start reading this layer's cache while the previous launch drains only if that
+    // launch was a decode step of another layer issued through this object on the same stream
+    const int early = (c->last_kind == 1 && c->last_layer != layer && c->last_stream == (void*)stream) ? 1 : 0;
+    e = buzz_launch_decode_bf16(c, layer, q, k_new, v_new, out, cs, early, stream);   // tensor-core kernel
+    if (e == cudaSuccess) { c->last_kind = 1; c->last_layer = layer; c->last_stream = (void*)stream; }
   } else {
     e = c->sh.head_dim == 128 ? launch_g<float, 128>(c, layer, q, k_new, v_new, out, cs, stream)
                               : launch_g<float, 64>(c, layer, q, k_new, v_new, out, cs, stream);
+    c->last_kind = 2;
   }
   if (e == cudaSuccess) c->launches += 1;
   return e;

@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(kThreads)
 decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict__ q,
                    const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
                    __nv_bfloat16* __restrict__ out, int layer, int max_batch, int kv_heads,
-                   int chunk_cap, float scale_log2, int logn) {
+                   int chunk_cap, float scale_log2, int logn, int early) {
   constexpr int NCH = D / 8;          // 16-byte chunks per row
   constexpr int KL = NCH / 4;         // K chunks per lane and row
   constexpr int VJ = NCH / 8;         // V chunks per lane and row
@@ -88,10 +88,16 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   float* owarp = invL + G;                                   // [kWarps][G][D]
   float* sl = owarp + kWarps * G * D;                        // [G][chunk_cap] logits (log2 domain)
 
-  // Programmatic dependent launch: let the next kernel in the stream begin its launch now, and do
-  // not touch global memory before everything earlier in the stream has completed and flushed.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Programmatic dependent launch. `early` is set by the host only when the kernel launched just
+  // before this one through the same object and stream was a decode step of ANOTHER layer: nothing
+  // it writes is read here before the wait, so this kernel may read its own layer's counters and
+  // pull its K and V rows towards L2 while that kernel drains. Otherwise it waits first.
+  // A kernel triggers its dependents only where its own pre-wait reads are safe to begin.
+  if (early) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  else {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
   const int n0 = st.n[inst];
   const int tot = st.total[inst];
   if (n0 >= pol.budget) {          // uniform over the cluster: every CTA read the same n0
@@ -111,6 +117,17 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   const uint4* Vc = reinterpret_cast<const uint4*>(st.V) + cache_off;
   const uint4* knew = reinterpret_cast<const uint4*>(k_new) + ((size_t)seq * kv_heads + head) * NCH;
   const uint4* vnew = reinterpret_cast<const uint4*>(v_new) + ((size_t)seq * kv_heads + head) * NCH;
+
+  if (early) {
+    const char* kb = reinterpret_cast<const char*>(Kc + (size_t)lo * NCH);
+    const char* vb = reinterpret_cast<const char*>(Vc + (size_t)lo * NCH);
+    const int lines = (cnt * NCH * 16) >> 7;                    // 128-byte lines of this CTA's K (and V) chunk
+    for (int i = tid; i < lines; i += kThreads) {
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(kb + (size_t)i * 128));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(vb + (size_t)i * 128));
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");         // q, k_new, v_new and out belong to the caller's chain
+  }
 
   // The CTA whose chunk holds slot n0 stores the appended token (Eq. 2).
   if (n0 >= lo && n0 < hi) {
@@ -315,7 +332,7 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
 
 template <int D, int G>
 cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, const void* v_new,
-                   void* out, int cluster_size, cudaStream_t stream) {
+                   void* out, int cluster_size, int early, cudaStream_t stream) {
   const int batch = c->batch[layer];
   const int chunk_cap = (((c->pol.budget + cluster_size - 1) / cluster_size + 1) & ~1) + 2;
   const size_t smem = sizeof(Partial<G, D>) +
@@ -346,17 +363,17 @@ cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, con
   return cudaLaunchKernelEx(&cfg, decode_bf16_kernel<D, G>, c->st, c->pol, (const __nv_bfloat16*)q,
                             (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, (__nv_bfloat16*)out,
                             layer, c->sh.max_batch, c->sh.kv_heads, chunk_cap, scale_log2,
-                            (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0);
+                            (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0, early);
 }
 
 template <int D>
 cudaError_t launch_g(buzz_ctx* c, int layer, const void* q, const void* k_new, const void* v_new,
-                     void* out, int cs, cudaStream_t stream) {
+                     void* out, int cs, int early, cudaStream_t stream) {
   switch (c->group) {
-    case 1: return launch<D, 1>(c, layer, q, k_new, v_new, out, cs, stream);
-    case 2: return launch<D, 2>(c, layer, q, k_new, v_new, out, cs, stream);
-    case 4: return launch<D, 4>(c, layer, q, k_new, v_new, out, cs, stream);
-    case 8: return launch<D, 8>(c, layer, q, k_new, v_new, out, cs, stream);
+    case 1: return launch<D, 1>(c, layer, q, k_new, v_new, out, cs, early, stream);
+    case 2: return launch<D, 2>(c, layer, q, k_new, v_new, out, cs, early, stream);
+    case 4: return launch<D, 4>(c, layer, q, k_new, v_new, out, cs, early, stream);
+    case 8: return launch<D, 8>(c, layer, q, k_new, v_new, out, cs, early, stream);
     default: return cudaErrorInvalidValue;
   }
 }
@@ -364,7 +381,7 @@ cudaError_t launch_g(buzz_ctx* c, int layer, const void* q, const void* k_new, c
 }  // namespace
 
 cudaError_t buzz_launch_decode_bf16(buzz_ctx* c, int layer, const void* q, const void* k_new,
-                                    const void* v_new, void* out, int cluster_size, cudaStream_t stream) {
-  return c->sh.head_dim == 128 ? launch_g<128>(c, layer, q, k_new, v_new, out, cluster_size, stream)
-                               : launch_g<64>(c, layer, q, k_new, v_new, out, cluster_size, stream);
+                                    const void* v_new, void* out, int cluster_size, int early, cudaStream_t stream) {
+  return c->sh.head_dim == 128 ? launch_g<128>(c, layer, q, k_new, v_new, out, cluster_size, early, stream)
+                               : launch_g<64>(c, layer, q, k_new, v_new, out, cluster_size, early, stream);
 }

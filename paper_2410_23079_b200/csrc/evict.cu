@@ -173,5 +173,6 @@ cudaError_t buzz_launch_evict(buzz_ctx* c, int layer_begin, int layer_count, cud
   }
 #undef BUZZ_EVICT_CASE
   c->launches += 1;
+  c->last_kind = 2;
   return cudaGetLastError();
 }

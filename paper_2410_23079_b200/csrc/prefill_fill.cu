@@ -141,5 +141,6 @@ cudaError_t buzz_launch_prefill_fill(buzz_ctx* c, int layer, const void* k, cons
   }
 #undef BUZZ_FILL_CASE
   c->launches += 1;
+  c->last_kind = 2;
   return cudaGetLastError();
 }
