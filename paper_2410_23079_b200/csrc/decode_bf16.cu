@@ -32,6 +32,7 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kMaxCluster = 8;
 constexpr int kHeads = 8;       // MMA column count: query heads of one group, zero-padded
 constexpr int kTile = 16;       // keys per warp tile
+constexpr int kPrefetchLines = 256;   // 128-byte lines of K a CTA may pull towards L2 before its wait (measured best)
 
 __device__ inline uint4 ld_stream(const uint4* p) { return __ldcs(p); }
 
@@ -91,7 +92,7 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   // Programmatic dependent launch. `early` is set by the host only when the kernel launched just
   // before this one through the same object and stream was a decode step of ANOTHER layer: nothing
   // it writes is read here before the wait, so this kernel may read its own layer's counters and
-  // pull its K and V rows towards L2 while that kernel drains. Otherwise it waits first.
+  // pull the head of its K rows towards L2 while that kernel drains. Otherwise it waits first.
   // A kernel triggers its dependents only where its own pre-wait reads are safe to begin.
   if (early) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   else {
@@ -120,11 +121,10 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
 
   if (early) {
     const char* kb = reinterpret_cast<const char*>(Kc + (size_t)lo * NCH);
-    const char* vb = reinterpret_cast<const char*>(Vc + (size_t)lo * NCH);
-    const int lines = (cnt * NCH * 16) >> 7;                    // 128-byte lines of this CTA's K (and V) chunk
+    // only the head of the chunk: enough to cover the start-up latency without flooding L2
+    const int lines = min((cnt * NCH * 16) >> 7, kPrefetchLines);
     for (int i = tid; i < lines; i += kThreads) {
       asm volatile("prefetch.global.L2 [%0];" ::"l"(kb + (size_t)i * 128));
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(vb + (size_t)i * 128));
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");         // q, k_new, v_new and out belong to the caller's chain
   }
