@@ -29,7 +29,6 @@ using namespace sm100;
 
 constexpr int D = 128;                    // head dim
 constexpr int BT = 128;                   // tile edge: query rows and keys per tile
-constexpr int kThreads = 192;
 constexpr uint32_t kBlockBytes = BT * 128;          // one [128 rows x 64 bf16] swizzled block
 constexpr uint32_t kTileBytes = 2 * kBlockBytes;    // a [128 x 128] bf16 tile = two blocks
 constexpr float kInvLn512 = 1.0f / 6.2383246250395077f;
@@ -88,8 +87,8 @@ __device__ __forceinline__ void colsum_tile(const uint32_t (&r)[NC], const float
 struct SmemB {
   alignas(1024) unsigned char k[kTileBytes];
   alignas(1024) unsigned char q[2][kTileBytes];
-  float lse[2][BT];
-  float rs[2][BT];
+  float lse[2][8][64];                     // [tile parity][compute warp][column of its half]: per-warp copies,
+  float rs[2][8][64];                      // so the compute warps never meet at a CTA-wide barrier inside the loop
   float part[BT];                          // warpgroup 1's partial column sums
   uint64_t k_full, q_full[2], q_empty[2], s_full[2], s_empty[2];
   uint32_t tmem_base;
@@ -169,24 +168,33 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int g = (warp - 2) >> 2;
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;              // TMEM lane = key within the tile
-    const int t = (warp - 2) * 32 + lane;             // 0..255 among the compute threads
     const int kpos = key0 + row;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};           // column c adds into acc[c % 4]: a fixed order
     bool ok = true;
+    // row statistics of tile `it` for this warp's 64 columns (two per lane): fetched from global
+    // memory one iteration ahead, so the load's latency hides behind the previous tile's exponentials
+    const int cw = warp - 2;                          // compute warp 0..7
+    auto fetch_lse = [&](int it, int e) -> float {
+      if (it >= iters) return 0.f;
+      const int qpos = (kt + it % nq) * BT + g * 64 + lane + 32 * e;
+      return (qpos < N) ? lse[(size_t)(kvh * G + it / nq) * stride + tok0 + qpos] : 0.f;
+    };
+    float lse_next0 = fetch_lse(0, 0), lse_next1 = fetch_lse(0, 1);
     for (int it = 0; it < iters; ++it) {
       const int st = it & 1, use = it >> 1;
-      const int gq = it / nq, qt = kt + it % nq;
+      const int qt = kt + it % nq;
       const int q0 = qt * BT;
-      const int h = kvh * G + gq;
-      // stage this tile's row statistics; the named barrier below publishes them
-      if (t < BT) {
-        const int qpos = q0 + t;
-        sm.lse[st][t] = (qpos < N) ? lse[(size_t)h * stride + tok0 + qpos] : 0.f;
-        sm.rs[st][t] = scale_log2 * (logn ? __logf((float)(qpos + 1)) * kInvLn512 : 1.0f);
+      // this warp's private copy of the tile's row statistics (last read two iterations ago by this warp only)
+      sm.lse[st][cw][lane] = lse_next0;
+      sm.lse[st][cw][lane + 32] = lse_next1;
+      if (logn) {
+        sm.rs[st][cw][lane] = scale_log2 * __logf((float)(q0 + g * 64 + lane + 1)) * kInvLn512;
+        sm.rs[st][cw][lane + 32] = scale_log2 * __logf((float)(q0 + g * 64 + lane + 33)) * kInvLn512;
       }
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      // (a thread that gave up on a wait keeps taking part in the named barriers, without waiting again)
-      if (ok && !mbar_wait(&sm.s_full[st], use & 1)) { tf.raise(5); ok = false; }
+      lse_next0 = fetch_lse(it + 1, 0);
+      lse_next1 = fetch_lse(it + 1, 1);
+      __syncwarp();
+      if (!mbar_wait(&sm.s_full[st], use & 1)) { tf.raise(5); ok = false; break; }
       tc_fence_after();
       const bool diag = (qt == kt), tail = (q0 + BT > N);
       // this thread's 64 logits first (two loads in flight), then 64 independent exponentials
@@ -196,10 +204,9 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(&sm.s_empty[st]);                    // S^T[st] may be overwritten once all 256 have arrived
-      if (logn) colsum_tile<true, 64>(r, sm.rs[st] + g * 64, sm.lse[st] + g * 64, scale_log2, diag, tail, q0 + g * 64, kpos, N, acc);
-      else colsum_tile<false, 64>(r, sm.rs[st] + g * 64, sm.lse[st] + g * 64, scale_log2, diag, tail, q0 + g * 64, kpos, N, acc);
-      // lse[st]/rs[st] are restaged two iterations from now; the named barrier of the next
-      // iteration, which every thread reaches only after these reads, orders that.
+      if (logn) colsum_tile<true, 64>(r, sm.rs[st][cw], sm.lse[st][cw], scale_log2, diag, tail, q0 + g * 64, kpos, N, acc);
+      else colsum_tile<false, 64>(r, sm.rs[st][cw], sm.lse[st][cw], scale_log2, diag, tail, q0 + g * 64, kpos, N, acc);
+      __syncwarp();                                   // the copy is rewritten two iterations from now
     }
     const float mine = (acc[0] + acc[1]) + (acc[2] + acc[3]);
     if (g == 1) sm.part[row] = mine;
