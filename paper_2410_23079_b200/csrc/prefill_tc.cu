@@ -230,17 +230,20 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 // warpgroups never synchronise inside the loop, so one can be taking maxima or waiting while the
 // other keeps the exponential unit busy; their (max, sum, output) are merged in the epilogue.
 //   TMEM columns: S0 [0,128)  S1 [128,256)  O_0 [256,384)  O_1 [384,512).
-// P_g (bf16 pairs, 32 columns) overwrites the start of the half row of S it was computed from.
-// The tensor core may still be reading P as the A operand long after the MMA was issued, so the
-// logits that reuse an S buffer are only issued once both P V products on it have been seen to
-// complete (pv_done).
+// P goes to SHARED memory (bf16, the K-major 128-byte-swizzled layout the MMA reads, written by
+// hand; half g of a row is row `row` of block g) and the P V products are shared x shared MMAs.
+// Keeping P out of tensor memory matters for latency, not capacity: if P shared columns with S, the
+// next logits into that buffer would have to wait for the P V product to complete (a tensor-core
+// read of its A operand is not ordered against a later MMA's writes), which puts
+// MMA -> commit -> wake-up -> MMA -> commit -> wake-up on the critical path of every tile.
 // =================================================================================================
 constexpr int kThreadsA = 320;            // TMA warp, MMA warp, 2 x 4 softmax warps
-constexpr int kStagesA = 3;
+constexpr int kStagesA = 2;
 struct SmemA {
   alignas(1024) unsigned char q[kTileBytes];
   alignas(1024) unsigned char k[kStagesA][kTileBytes];
   alignas(1024) unsigned char v[kStagesA][kTileBytes];
+  alignas(1024) unsigned char p[2][kTileBytes];      // [tile parity]: block g = warpgroup g's 64 key columns
   uint64_t q_full, k_full[kStagesA], k_empty[kStagesA], v_full[kStagesA], v_empty[kStagesA];
   uint64_t s_full[2], p_full[2][2], pv_done[2];
   uint32_t tmem_base;
@@ -326,21 +329,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (!ok) tf.raise(14);
       ok = ok && issue_qk(0);
       for (int j = 0; ok && j < nt; ++j) {
-        if (j + 1 < nt) {
-          // S[(j+1)%2] still holds P of tile j-1: both of its P V products must have completed
-          if (j >= 1 && !mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(21); break; }
-          if (!issue_qk(j + 1)) break;                 // next tile's logits overlap this tile's softmax
-        }
+        // S[(j+1)%2] was last read by the softmax of tile j-1, which has arrived on p_full(j-1)
+        if (j + 1 < nt && !issue_qk(j + 1)) break;     // next tile's logits overlap this tile's softmax
         const int sb = j & 1, st = j % kStagesA;
         bool fine = true;
         for (int g = 0; g < 2 && fine; ++g) {          // O_g += P_g V[64g .. 64g+63], 16 keys per step
           if (!mbar_wait(&sm.p_full[sb][g], (j >> 1) & 1)) { tf.raise(15); fine = false; break; }
           if (g == 0 && !mbar_wait(&sm.v_full[st], (j / kStagesA) & 1)) { tf.raise(16); fine = false; break; }
           tc_fence_after();
-          const uint32_t va = smem_u32(sm.v[st]);
+          const uint32_t va = smem_u32(sm.v[st]), pa = smem_u32(sm.p[sb]);
 #pragma unroll
           for (int s = 0; s < 4; ++s)
-            mma_ts(tmem + kColO + g * BT, tmem + sb * BT + g * 64 + s * 8, mnmajor_desc(va, g * 4 + s), kIdescKM,
+            mma_ss(tmem + kColO + g * BT, kmajor_desc(pa, g * 4 + s), mnmajor_desc(va, g * 4 + s), kIdescKM,
                    (j > 0 || s > 0) ? 1u : 0u);
         }
         if (!fine) break;
@@ -401,22 +401,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           tmem_wait_st();
         }
       }
-      // P_g = 2^(S rs - m) as bf16 pairs over the first 32 columns of this half row (which is in registers)
+      // P_g = 2^(S rs - m) as bf16 into row `row` of block g of P[sb], once the P V products of
+      // tile j-2 have consumed that buffer
+      if (j >= 2 && !mbar_wait(&sm.pv_done[sb], ((j >> 1) - 1) & 1)) { tf.raise(20); ok = false; break; }
       const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
       float l4[4] = {0.f, 0.f, 0.f, 0.f};
-      uint32_t pk[32];
+      unsigned char* prow = sm.p[sb] + g * kBlockBytes + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
-      for (int c = 0; c < 32; ++c) {
-        const float p0 = exp2f(fmaf(s[2 * c], rs, neg_m));
-        const float p1 = exp2f(fmaf(s[2 * c + 1], rs, neg_m));
-        l4[c & 3] += p0 + p1;
-        const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
-        pk[c] = *reinterpret_cast<const uint32_t*>(&pp);
+      for (int ch = 0; ch < 8; ++ch) {                 // 16-byte chunk ch = keys 8 ch .. 8 ch + 7 of this half
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float p0 = exp2f(fmaf(s[ch * 8 + 2 * e], rs, neg_m));
+          const float p1 = exp2f(fmaf(s[ch * 8 + 2 * e + 1], rs, neg_m));
+          l4[e] += p0 + p1;
+          const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
+          w[e] = *reinterpret_cast<const uint32_t*>(&pp);
+        }
+        *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
       }
-      tmem_st32(tmem + lane_base + colS, pk);
       l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
-      tmem_wait_st();
-      tc_fence_before();
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
+      tc_fence_before();                               // this thread's TMEM loads (and rescale stores) are done
       mbar_arrive(&sm.p_full[sb][g]);
     }
     // ---- epilogue: merge the two halves of the row, O / l -> bf16, row log2-sum-exp ----
