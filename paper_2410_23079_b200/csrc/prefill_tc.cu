@@ -237,14 +237,14 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 // read of its A operand is not ordered against a later MMA's writes), which puts
 // MMA -> commit -> wake-up -> MMA -> commit -> wake-up on the critical path of every tile.
 // =================================================================================================
-constexpr int kThreadsA = 320;            // TMA warp, MMA warp, 2 x 4 softmax warps
-constexpr int kStagesA = 2;
+constexpr int kThreadsA = 352;            // K/Q TMA warp, MMA warp, 2 x 4 softmax warps, V TMA warp
+constexpr int kStagesK = 3, kStagesV = 2; // a tile takes ~2000 cycles to arrive: K is needed a tile earlier than V
 struct SmemA {
   alignas(1024) unsigned char q[kTileBytes];
-  alignas(1024) unsigned char k[kStagesA][kTileBytes];
-  alignas(1024) unsigned char v[kStagesA][kTileBytes];
-  alignas(1024) unsigned char p[2][kTileBytes];      // [tile parity]: block g = warpgroup g's 64 key columns
-  uint64_t q_full, k_full[kStagesA], k_empty[kStagesA], v_full[kStagesA], v_empty[kStagesA];
+  alignas(1024) unsigned char k[kStagesK][kTileBytes];
+  alignas(1024) unsigned char v[kStagesV][kTileBytes];
+  alignas(1024) unsigned char p[kTileBytes];         // block g = warpgroup g's 64 key columns
+  uint64_t q_full, k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
   uint64_t s_full[2], p_full[2][2], pv_done[2];
   uint32_t tmem_base;
 };
@@ -274,10 +274,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
   if (threadIdx.x == 0) {
     mbar_init(&sm.q_full, 1);
-    for (int s = 0; s < kStagesA; ++s) {
-      mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1);
-      mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
-    }
+    for (int s = 0; s < kStagesK; ++s) { mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1); }
+    for (int s = 0; s < kStagesV; ++s) { mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1); }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sm.s_full[s], 1); mbar_init(&sm.pv_done[s], 1);
       mbar_init(&sm.p_full[s][0], 128); mbar_init(&sm.p_full[s][1], 128);
@@ -300,10 +298,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_expect_tx(&sm.q_full, kTileBytes);
       load_tile(sm.q, &map_q, h * D, tok0 + row0, &sm.q_full);
       for (int j = 0; j < nt; ++j) {
-        const int st = j % kStagesA, use = j / kStagesA;
+        const int st = j % kStagesK, use = j / kStagesK;
         if (use > 0 && !mbar_wait(&sm.k_empty[st], (use - 1) & 1)) { tf.raise(11); break; }
         mbar_expect_tx(&sm.k_full[st], kTileBytes);
         load_tile(sm.k[st], &map_k, kvh * D, tok0 + j * BT, &sm.k_full[st]);
+      }
+    }
+  } else if (warp == 10) {
+    // ---- TMA producer for V (its own warp: a full V ring must not hold back the K loads) ----
+    if (elect_one()) {
+      for (int j = 0; j < nt; ++j) {
+        const int st = j % kStagesV, use = j / kStagesV;
         if (use > 0 && !mbar_wait(&sm.v_empty[st], (use - 1) & 1)) { tf.raise(12); break; }
         mbar_expect_tx(&sm.v_full[st], kTileBytes);
         load_tile(sm.v[st], &map_v, kvh * D, tok0 + j * BT, &sm.v_full[st]);
@@ -314,8 +319,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (elect_one()) {
       const uint32_t qa = smem_u32(sm.q);
       auto issue_qk = [&](int j) -> bool {             // S[j%2] = Q K_j^T
-        const int st = j % kStagesA;
-        if (!mbar_wait(&sm.k_full[st], (j / kStagesA) & 1)) { tf.raise(13); return false; }
+        const int st = j % kStagesK;
+        if (!mbar_wait(&sm.k_full[st], (j / kStagesK) & 1)) { tf.raise(13); return false; }
         tc_fence_after();
         const uint32_t ka = smem_u32(sm.k[st]);
 #pragma unroll
@@ -331,13 +336,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       for (int j = 0; ok && j < nt; ++j) {
         // S[(j+1)%2] was last read by the softmax of tile j-1, which has arrived on p_full(j-1)
         if (j + 1 < nt && !issue_qk(j + 1)) break;     // next tile's logits overlap this tile's softmax
-        const int sb = j & 1, st = j % kStagesA;
+        const int sb = j & 1, st = j % kStagesV;
         bool fine = true;
         for (int g = 0; g < 2 && fine; ++g) {          // O_g += P_g V[64g .. 64g+63], 16 keys per step
           if (!mbar_wait(&sm.p_full[sb][g], (j >> 1) & 1)) { tf.raise(15); fine = false; break; }
-          if (g == 0 && !mbar_wait(&sm.v_full[st], (j / kStagesA) & 1)) { tf.raise(16); fine = false; break; }
+          if (g == 0 && !mbar_wait(&sm.v_full[st], (j / kStagesV) & 1)) { tf.raise(16); fine = false; break; }
           tc_fence_after();
-          const uint32_t va = smem_u32(sm.v[st]), pa = smem_u32(sm.p[sb]);
+          const uint32_t va = smem_u32(sm.v[st]), pa = smem_u32(sm.p);
 #pragma unroll
           for (int s = 0; s < 4; ++s)
             mma_ss(tmem + kColO + g * BT, kmajor_desc(pa, g * 4 + s), mnmajor_desc(va, g * 4 + s), kIdescKM,
@@ -350,7 +355,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
   } else {
     // ---- softmax: thread (g, row) runs an online softmax over key columns [64g, 64g+64) of every tile ----
-    const int g = (warp - 2) >> 2;
+    const int g = (warp - 2) >> 2;    // warps 2..9
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const int qpos = row0 + row;
@@ -401,12 +406,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           tmem_wait_st();
         }
       }
-      // P_g = 2^(S rs - m) as bf16 into row `row` of block g of P[sb], once the P V products of
-      // tile j-2 have consumed that buffer
-      if (j >= 2 && !mbar_wait(&sm.pv_done[sb], ((j >> 1) - 1) & 1)) { tf.raise(20); ok = false; break; }
+      // P_g = 2^(S rs - m) as bf16 into row `row` of block g of P, once the P V products of tile j-1
+      // have consumed it (they were issued a whole softmax ago)
+      if (j >= 1 && !mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(20); ok = false; break; }
       const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
       float l4[4] = {0.f, 0.f, 0.f, 0.f};
-      unsigned char* prow = sm.p[sb] + g * kBlockBytes + (row >> 3) * 1024 + (row & 7) * 128;
+      unsigned char* prow = sm.p + g * kBlockBytes + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
       for (int ch = 0; ch < 8; ++ch) {                 // 16-byte chunk ch = keys 8 ch .. 8 ch + 7 of this half
         uint32_t w[4];
