@@ -238,12 +238,12 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 // MMA -> commit -> wake-up -> MMA -> commit -> wake-up on the critical path of every tile.
 // =================================================================================================
 constexpr int kThreadsA = 352;            // K/Q TMA warp, MMA warp, 2 x 4 softmax warps, V TMA warp
-constexpr int kStagesK = 3, kStagesV = 2; // a tile takes ~2000 cycles to arrive: K is needed a tile earlier than V
+constexpr int kStagesK = 2, kStagesV = 2; // each ring has its own producer warp, so a full V ring never delays K
 struct SmemA {
   alignas(1024) unsigned char q[kTileBytes];
   alignas(1024) unsigned char k[kStagesK][kTileBytes];
   alignas(1024) unsigned char v[kStagesV][kTileBytes];
-  alignas(1024) unsigned char p[kTileBytes];         // block g = warpgroup g's 64 key columns
+  alignas(1024) unsigned char p[2][kTileBytes];      // [tile parity]: block g = warpgroup g's 64 key columns
   uint64_t q_full, k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
   uint64_t s_full[2], p_full[2][2], pv_done[2];
   uint32_t tmem_base;
@@ -342,7 +342,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           if (!mbar_wait(&sm.p_full[sb][g], (j >> 1) & 1)) { tf.raise(15); fine = false; break; }
           if (g == 0 && !mbar_wait(&sm.v_full[st], (j / kStagesV) & 1)) { tf.raise(16); fine = false; break; }
           tc_fence_after();
-          const uint32_t va = smem_u32(sm.v[st]), pa = smem_u32(sm.p);
+          const uint32_t va = smem_u32(sm.v[st]), pa = smem_u32(sm.p[sb]);
 #pragma unroll
           for (int s = 0; s < 4; ++s)
             mma_ss(tmem + kColO + g * BT, kmajor_desc(pa, g * 4 + s), mnmajor_desc(va, g * 4 + s), kIdescKM,
@@ -406,12 +406,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           tmem_wait_st();
         }
       }
-      // P_g = 2^(S rs - m) as bf16 into row `row` of block g of P, once the P V products of tile j-1
-      // have consumed it (they were issued a whole softmax ago)
-      if (j >= 1 && !mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(20); ok = false; break; }
+      // P_g = 2^(S rs - m) as bf16 into row `row` of block g of P[sb], once the P V products of
+      // tile j-2 have consumed that buffer
+      if (j >= 2 && !mbar_wait(&sm.pv_done[sb], ((j >> 1) - 1) & 1)) { tf.raise(20); ok = false; break; }
       const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
       float l4[4] = {0.f, 0.f, 0.f, 0.f};
-      unsigned char* prow = sm.p + g * kBlockBytes + (row >> 3) * 1024 + (row & 7) * 128;
+      unsigned char* prow = sm.p[sb] + g * kBlockBytes + (row >> 3) * 1024 + (row & 7) * 128;
 #pragma unroll
       for (int ch = 0; ch < 8; ++ch) {                 // 16-byte chunk ch = keys 8 ch .. 8 ch + 7 of this half
         uint32_t w[4];
