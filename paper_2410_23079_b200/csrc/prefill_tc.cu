@@ -333,9 +333,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       bool ok = mbar_wait(&sm.q_full, 0);
       if (!ok) tf.raise(14);
       ok = ok && issue_qk(0);
+      if (ok && nt > 1) ok = issue_qk(1);
       for (int j = 0; ok && j < nt; ++j) {
-        // S[(j+1)%2] was last read by the softmax of tile j-1, which has arrived on p_full(j-1)
-        if (j + 1 < nt && !issue_qk(j + 1)) break;     // next tile's logits overlap this tile's softmax
         const int sb = j & 1, st = j % kStagesV;
         bool fine = true;
         for (int g = 0; g < 2 && fine; ++g) {          // O_g += P_g V[64g .. 64g+63], 16 keys per step
@@ -351,6 +350,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         if (!fine) break;
         mma_commit(&sm.v_empty[st]);
         mma_commit(&sm.pv_done[sb]);
+        // S[sb] was read into registers by the softmax of tile j before it arrived on p_full(j): the
+        // logits of tile j+2 can go there now, two tiles ahead of their softmax
+        if (j + 2 < nt && !issue_qk(j + 2)) break;
       }
     }
   } else {
