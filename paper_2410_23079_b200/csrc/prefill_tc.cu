@@ -34,6 +34,7 @@ constexpr uint32_t kTileBytes = 2 * kBlockBytes;    // a [128 x 128] bf16 tile =
 constexpr float kInvLn512 = 1.0f / 6.2383246250395077f;
 constexpr uint32_t kIdescKK = idesc_bf16(BT, BT, false, false);   // both operands K-major
 constexpr uint32_t kIdescKM = idesc_bf16(BT, BT, false, true);    // B operand MN-major (V)
+constexpr uint32_t kIdescKK64 = idesc_bf16(BT, 64, false, false); // logits of 64 keys
 
 struct TimeoutFlag {
   int32_t* status;
@@ -245,10 +246,11 @@ struct SmemA {
   alignas(1024) unsigned char v[kStagesV][kTileBytes];
   alignas(1024) unsigned char p[2][kTileBytes];      // [tile parity]: block g = warpgroup g's 64 key columns
   uint64_t q_full, k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
-  uint64_t s_full[2], p_full[2][2], pv_done[2];
+  uint64_t s_full[2][2], p_full[2][2], pv_done[2][2];   // [tile parity][warpgroup]
   uint32_t tmem_base;
 };
 constexpr uint32_t kColO = 256;
+constexpr long long kStreamSkewCycles = 700;
 constexpr float kRescaleThreshold = 20.0f;    // log2: rescale O only when a row max grows by > 2^20
                                               // (P, the row sums and O stay far inside the fp32/bf16 exponent range)
 
@@ -277,8 +279,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     for (int s = 0; s < kStagesK; ++s) { mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1); }
     for (int s = 0; s < kStagesV; ++s) { mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1); }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&sm.s_full[s], 1); mbar_init(&sm.pv_done[s], 1);
-      mbar_init(&sm.p_full[s][0], 128); mbar_init(&sm.p_full[s][1], 128);
+      for (int g2 = 0; g2 < 2; ++g2) {
+        mbar_init(&sm.s_full[s][g2], 1); mbar_init(&sm.pv_done[s][g2], 1); mbar_init(&sm.p_full[s][g2], 128);
+      }
     }
     fence_barrier_init();
   }
@@ -318,41 +321,46 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // ---- MMA issuer ----
     if (elect_one()) {
       const uint32_t qa = smem_u32(sm.q);
-      auto issue_qk = [&](int j) -> bool {             // S[j%2] = Q K_j^T
-        const int st = j % kStagesK;
-        if (!mbar_wait(&sm.k_full[st], (j / kStagesK) & 1)) { tf.raise(13); return false; }
-        tc_fence_after();
-        const uint32_t ka = smem_u32(sm.k[st]);
+      // Two independent streams, one per softmax warpgroup g: logits S_g = Q K_j[64g..64g+63]^T (N = 64),
+      // and O_g += P_g V_j[64g..64g+63]. A stream's logits for tile j+2 are issued right after its
+      // P V product of tile j: S_g[j%2] was read into registers before the warpgroup arrived on p_full.
+      auto issue_qk = [&](int j, int g) -> void {
+        const uint32_t ka = smem_u32(sm.k[j % kStagesK]) + g * 64 * 128;   // key rows 64g.. of both dim blocks
 #pragma unroll
         for (int s = 0; s < D / 16; ++s)
-          mma_ss(tmem + (j & 1) * BT, kmajor_desc(qa, s), kmajor_desc(ka, s), kIdescKK, s > 0);
-        mma_commit(&sm.s_full[j & 1]);
-        mma_commit(&sm.k_empty[st]);
-        return true;
+          mma_ss(tmem + (j & 1) * BT + g * 64, kmajor_desc(qa, s), kmajor_desc(ka, s), kIdescKK64, s > 0);
+        mma_commit(&sm.s_full[j & 1][g]);
+        if (g == 1) mma_commit(&sm.k_empty[j % kStagesK]);
+      };
+      auto wait_k = [&](int j) -> bool {
+        if (mbar_wait(&sm.k_full[j % kStagesK], (j / kStagesK) & 1)) { tc_fence_after(); return true; }
+        tf.raise(13);
+        return false;
       };
       bool ok = mbar_wait(&sm.q_full, 0);
       if (!ok) tf.raise(14);
-      ok = ok && issue_qk(0);
-      if (ok && nt > 1) ok = issue_qk(1);
+      for (int j = 0; ok && j < 2 && j < nt; ++j) {
+        ok = wait_k(j);
+        if (ok) { issue_qk(j, 0); issue_qk(j, 1); }
+      }
       for (int j = 0; ok && j < nt; ++j) {
         const int sb = j & 1, st = j % kStagesV;
-        bool fine = true;
-        for (int g = 0; g < 2 && fine; ++g) {          // O_g += P_g V[64g .. 64g+63], 16 keys per step
-          if (!mbar_wait(&sm.p_full[sb][g], (j >> 1) & 1)) { tf.raise(15); fine = false; break; }
-          if (g == 0 && !mbar_wait(&sm.v_full[st], (j / kStagesV) & 1)) { tf.raise(16); fine = false; break; }
+        for (int g = 0; g < 2 && ok; ++g) {
+          if (!mbar_wait(&sm.p_full[sb][g], (j >> 1) & 1)) { tf.raise(15); ok = false; break; }
+          if (g == 0 && !mbar_wait(&sm.v_full[st], (j / kStagesV) & 1)) { tf.raise(16); ok = false; break; }
           tc_fence_after();
           const uint32_t va = smem_u32(sm.v[st]), pa = smem_u32(sm.p[sb]);
 #pragma unroll
-          for (int s = 0; s < 4; ++s)
+          for (int s = 0; s < 4; ++s)                  // O_g += P_g V[64g .. 64g+63], 16 keys per step
             mma_ss(tmem + kColO + g * BT, kmajor_desc(pa, g * 4 + s), mnmajor_desc(va, g * 4 + s), kIdescKM,
                    (j > 0 || s > 0) ? 1u : 0u);
+          mma_commit(&sm.pv_done[sb][g]);
+          if (g == 1) mma_commit(&sm.v_empty[st]);
+          if (j + 2 < nt) {
+            if (g == 0 && !wait_k(j + 2)) { ok = false; break; }
+            issue_qk(j + 2, g);
+          }
         }
-        if (!fine) break;
-        mma_commit(&sm.v_empty[st]);
-        mma_commit(&sm.pv_done[sb]);
-        // S[sb] was read into registers by the softmax of tile j before it arrived on p_full(j): the
-        // logits of tile j+2 can go there now, two tiles ahead of their softmax
-        if (j + 2 < nt && !issue_qk(j + 2)) break;
       }
     }
   } else {
@@ -366,10 +374,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const float rs = scale_log2 * (logn ? __logf((float)(qpos + 1)) * kInvLn512 : 1.0f);
     float m_used = -INFINITY, l = 0.f;
     bool ok = true;
+    if (g == 1) {                                      // start the second stream about half a tile late, so the two
+      const long long t0 = clock64();                  // warpgroups use the exponential unit in turns rather than together
+      while (clock64() - t0 < kStreamSkewCycles) { }
+    }
     for (int j = 0; j < nt; ++j) {
       const int sb = j & 1;
       const uint32_t colS = sb * BT + g * 64;
-      if (!mbar_wait(&sm.s_full[sb], (j >> 1) & 1)) { tf.raise(17); ok = false; break; }
+      if (!mbar_wait(&sm.s_full[sb][g], (j >> 1) & 1)) { tf.raise(17); ok = false; break; }
       tc_fence_after();
       // the raw logits of this half row (rs > 0, so the maximum can be taken before scaling)
       float s[64];
@@ -394,7 +406,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           const float alpha = need ? exp2f(m_used - m_new) : 1.0f;     // 0 when nothing was unmasked so far
           if (need) m_used = m_new;
           l *= alpha;
-          if (!mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
+          if (!mbar_wait(&sm.pv_done[(j - 1) & 1][g], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
           tc_fence_after();
 #pragma unroll 1
           for (int c0 = 0; c0 < D; c0 += 32) {
@@ -410,7 +422,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
       // P_g = 2^(S rs - m) as bf16 into row `row` of block g of P[sb], once the P V products of
       // tile j-2 have consumed that buffer
-      if (j >= 2 && !mbar_wait(&sm.pv_done[sb], ((j >> 1) - 1) & 1)) { tf.raise(20); ok = false; break; }
+      if (j >= 2 && !mbar_wait(&sm.pv_done[sb][g], ((j >> 1) - 1) & 1)) { tf.raise(20); ok = false; break; }
       const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
       float l4[4] = {0.f, 0.f, 0.f, 0.f};
       unsigned char* prow = sm.p[sb] + g * kBlockBytes + (row >> 3) * 1024 + (row & 7) * 128;
@@ -433,7 +445,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_arrive(&sm.p_full[sb][g]);
     }
     // ---- epilogue: merge the two halves of the row, O / l -> bf16, row log2-sum-exp ----
-    if (ok && !mbar_wait(&sm.pv_done[(nt - 1) & 1], ((nt - 1) >> 1) & 1)) { tf.raise(19); ok = false; }
+    if (ok && !(mbar_wait(&sm.pv_done[(nt - 1) & 1][0], ((nt - 1) >> 1) & 1) &&
+                mbar_wait(&sm.pv_done[(nt - 1) & 1][1], ((nt - 1) >> 1) & 1))) { tf.raise(19); ok = false; }
     tc_fence_after();
     // the K ring is idle now (its last use completed before that P V product): exchange (max, sum) there
     float* xm = reinterpret_cast<float*>(sm.k[0]);    // [2][BT]
