@@ -34,7 +34,6 @@ constexpr uint32_t kTileBytes = 2 * kBlockBytes;    // a [128 x 128] bf16 tile =
 constexpr float kInvLn512 = 1.0f / 6.2383246250395077f;
 constexpr uint32_t kIdescKK = idesc_bf16(BT, BT, false, false);   // both operands K-major
 constexpr uint32_t kIdescKM = idesc_bf16(BT, BT, false, true);    // B operand MN-major (V)
-constexpr uint32_t kIdescKK64 = idesc_bf16(BT, 64, false, false); // logits of 64 keys
 
 struct TimeoutFlag {
   int32_t* status;
@@ -231,26 +230,22 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 // warpgroups never synchronise inside the loop, so one can be taking maxima or waiting while the
 // other keeps the exponential unit busy; their (max, sum, output) are merged in the epilogue.
 //   TMEM columns: S0 [0,128)  S1 [128,256)  O_0 [256,384)  O_1 [384,512).
-// P goes to SHARED memory (bf16, the K-major 128-byte-swizzled layout the MMA reads, written by
-// hand; half g of a row is row `row` of block g) and the P V products are shared x shared MMAs.
-// Keeping P out of tensor memory matters for latency, not capacity: if P shared columns with S, the
-// next logits into that buffer would have to wait for the P V product to complete (a tensor-core
-// read of its A operand is not ordered against a later MMA's writes), which puts
-// MMA -> commit -> wake-up -> MMA -> commit -> wake-up on the critical path of every tile.
+// P_g (bf16 pairs, 32 columns) overwrites the start of the half row of S it was computed from.
+// The tensor core may still be reading P as the A operand long after the MMA was issued, so the
+// logits that reuse an S buffer are only issued once both P V products on it have been seen to
+// complete (pv_done).
 // =================================================================================================
-constexpr int kThreadsA = 352;            // K/Q TMA warp, MMA warp, 2 x 4 softmax warps, V TMA warp
-constexpr int kStagesK = 2, kStagesV = 2; // each ring has its own producer warp, so a full V ring never delays K
+constexpr int kThreadsA = 320;            // TMA warp, MMA warp, 2 x 4 softmax warps
+constexpr int kStagesA = 3;
 struct SmemA {
   alignas(1024) unsigned char q[kTileBytes];
-  alignas(1024) unsigned char k[kStagesK][kTileBytes];
-  alignas(1024) unsigned char v[kStagesV][kTileBytes];
-  alignas(1024) unsigned char p[2][kTileBytes];      // [tile parity]: block g = warpgroup g's 64 key columns
-  uint64_t q_full, k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
-  uint64_t s_full[2][2], p_full[2][2], pv_done[2][2];   // [tile parity][warpgroup]
+  alignas(1024) unsigned char k[kStagesA][kTileBytes];
+  alignas(1024) unsigned char v[kStagesA][kTileBytes];
+  uint64_t q_full, k_full[kStagesA], k_empty[kStagesA], v_full[kStagesA], v_empty[kStagesA];
+  uint64_t s_full[2], p_full[2][2], pv_done[2];
   uint32_t tmem_base;
 };
 constexpr uint32_t kColO = 256;
-constexpr long long kStreamSkewCycles = 700;
 constexpr float kRescaleThreshold = 20.0f;    // log2: rescale O only when a row max grows by > 2^20
                                               // (P, the row sums and O stay far inside the fp32/bf16 exponent range)
 
@@ -276,12 +271,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 
   if (threadIdx.x == 0) {
     mbar_init(&sm.q_full, 1);
-    for (int s = 0; s < kStagesK; ++s) { mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1); }
-    for (int s = 0; s < kStagesV; ++s) { mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1); }
+    for (int s = 0; s < kStagesA; ++s) {
+      mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1);
+      mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
+    }
     for (int s = 0; s < 2; ++s) {
-      for (int g2 = 0; g2 < 2; ++g2) {
-        mbar_init(&sm.s_full[s][g2], 1); mbar_init(&sm.pv_done[s][g2], 1); mbar_init(&sm.p_full[s][g2], 128);
-      }
+      mbar_init(&sm.s_full[s], 1); mbar_init(&sm.pv_done[s], 1);
+      mbar_init(&sm.p_full[s][0], 128); mbar_init(&sm.p_full[s][1], 128);
     }
     fence_barrier_init();
   }
@@ -301,17 +297,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_expect_tx(&sm.q_full, kTileBytes);
       load_tile(sm.q, &map_q, h * D, tok0 + row0, &sm.q_full);
       for (int j = 0; j < nt; ++j) {
-        const int st = j % kStagesK, use = j / kStagesK;
+        const int st = j % kStagesA, use = j / kStagesA;
         if (use > 0 && !mbar_wait(&sm.k_empty[st], (use - 1) & 1)) { tf.raise(11); break; }
         mbar_expect_tx(&sm.k_full[st], kTileBytes);
         load_tile(sm.k[st], &map_k, kvh * D, tok0 + j * BT, &sm.k_full[st]);
-      }
-    }
-  } else if (warp == 10) {
-    // ---- TMA producer for V (its own warp: a full V ring must not hold back the K loads) ----
-    if (elect_one()) {
-      for (int j = 0; j < nt; ++j) {
-        const int st = j % kStagesV, use = j / kStagesV;
         if (use > 0 && !mbar_wait(&sm.v_empty[st], (use - 1) & 1)) { tf.raise(12); break; }
         mbar_expect_tx(&sm.v_full[st], kTileBytes);
         load_tile(sm.v[st], &map_v, kvh * D, tok0 + j * BT, &sm.v_full[st]);
@@ -321,51 +310,47 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     // ---- MMA issuer ----
     if (elect_one()) {
       const uint32_t qa = smem_u32(sm.q);
-      // Two independent streams, one per softmax warpgroup g: logits S_g = Q K_j[64g..64g+63]^T (N = 64),
-      // and O_g += P_g V_j[64g..64g+63]. A stream's logits for tile j+2 are issued right after its
-      // P V product of tile j: S_g[j%2] was read into registers before the warpgroup arrived on p_full.
-      auto issue_qk = [&](int j, int g) -> void {
-        const uint32_t ka = smem_u32(sm.k[j % kStagesK]) + g * 64 * 128;   // key rows 64g.. of both dim blocks
+      auto issue_qk = [&](int j) -> bool {             // S[j%2] = Q K_j^T
+        const int st = j % kStagesA;
+        if (!mbar_wait(&sm.k_full[st], (j / kStagesA) & 1)) { tf.raise(13); return false; }
+        tc_fence_after();
+        const uint32_t ka = smem_u32(sm.k[st]);
 #pragma unroll
         for (int s = 0; s < D / 16; ++s)
-          mma_ss(tmem + (j & 1) * BT + g * 64, kmajor_desc(qa, s), kmajor_desc(ka, s), kIdescKK64, s > 0);
-        mma_commit(&sm.s_full[j & 1][g]);
-        if (g == 1) mma_commit(&sm.k_empty[j % kStagesK]);
-      };
-      auto wait_k = [&](int j) -> bool {
-        if (mbar_wait(&sm.k_full[j % kStagesK], (j / kStagesK) & 1)) { tc_fence_after(); return true; }
-        tf.raise(13);
-        return false;
+          mma_ss(tmem + (j & 1) * BT, kmajor_desc(qa, s), kmajor_desc(ka, s), kIdescKK, s > 0);
+        mma_commit(&sm.s_full[j & 1]);
+        mma_commit(&sm.k_empty[st]);
+        return true;
       };
       bool ok = mbar_wait(&sm.q_full, 0);
       if (!ok) tf.raise(14);
-      for (int j = 0; ok && j < 2 && j < nt; ++j) {
-        ok = wait_k(j);
-        if (ok) { issue_qk(j, 0); issue_qk(j, 1); }
-      }
+      ok = ok && issue_qk(0);
       for (int j = 0; ok && j < nt; ++j) {
-        const int sb = j & 1, st = j % kStagesV;
-        for (int g = 0; g < 2 && ok; ++g) {
-          if (!mbar_wait(&sm.p_full[sb][g], (j >> 1) & 1)) { tf.raise(15); ok = false; break; }
-          if (g == 0 && !mbar_wait(&sm.v_full[st], (j / kStagesV) & 1)) { tf.raise(16); ok = false; break; }
-          tc_fence_after();
-          const uint32_t va = smem_u32(sm.v[st]), pa = smem_u32(sm.p[sb]);
-#pragma unroll
-          for (int s = 0; s < 4; ++s)                  // O_g += P_g V[64g .. 64g+63], 16 keys per step
-            mma_ss(tmem + kColO + g * BT, kmajor_desc(pa, g * 4 + s), mnmajor_desc(va, g * 4 + s), kIdescKM,
-                   (j > 0 || s > 0) ? 1u : 0u);
-          mma_commit(&sm.pv_done[sb][g]);
-          if (g == 1) mma_commit(&sm.v_empty[st]);
-          if (j + 2 < nt) {
-            if (g == 0 && !wait_k(j + 2)) { ok = false; break; }
-            issue_qk(j + 2, g);
-          }
+        if (j + 1 < nt) {
+          // S[(j+1)%2] still holds P of tile j-1: both of its P V products must have completed
+          if (j >= 1 && !mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(21); break; }
+          if (!issue_qk(j + 1)) break;                 // next tile's logits overlap this tile's softmax
         }
+        const int sb = j & 1, st = j % kStagesA;
+        bool fine = true;
+        for (int g = 0; g < 2 && fine; ++g) {          // O_g += P_g V[64g .. 64g+63], 16 keys per step
+          if (!mbar_wait(&sm.p_full[sb][g], (j >> 1) & 1)) { tf.raise(15); fine = false; break; }
+          if (g == 0 && !mbar_wait(&sm.v_full[st], (j / kStagesA) & 1)) { tf.raise(16); fine = false; break; }
+          tc_fence_after();
+          const uint32_t va = smem_u32(sm.v[st]);
+#pragma unroll
+          for (int s = 0; s < 4; ++s)
+            mma_ts(tmem + kColO + g * BT, tmem + sb * BT + g * 64 + s * 8, mnmajor_desc(va, g * 4 + s), kIdescKM,
+                   (j > 0 || s > 0) ? 1u : 0u);
+        }
+        if (!fine) break;
+        mma_commit(&sm.v_empty[st]);
+        mma_commit(&sm.pv_done[sb]);
       }
     }
   } else {
     // ---- softmax: thread (g, row) runs an online softmax over key columns [64g, 64g+64) of every tile ----
-    const int g = (warp - 2) >> 2;    // warps 2..9
+    const int g = (warp - 2) >> 2;
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const int qpos = row0 + row;
@@ -374,14 +359,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const float rs = scale_log2 * (logn ? __logf((float)(qpos + 1)) * kInvLn512 : 1.0f);
     float m_used = -INFINITY, l = 0.f;
     bool ok = true;
-    if (g == 1) {                                      // start the second stream about half a tile late, so the two
-      const long long t0 = clock64();                  // warpgroups use the exponential unit in turns rather than together
-      while (clock64() - t0 < kStreamSkewCycles) { }
-    }
     for (int j = 0; j < nt; ++j) {
       const int sb = j & 1;
       const uint32_t colS = sb * BT + g * 64;
-      if (!mbar_wait(&sm.s_full[sb][g], (j >> 1) & 1)) { tf.raise(17); ok = false; break; }
+      if (!mbar_wait(&sm.s_full[sb], (j >> 1) & 1)) { tf.raise(17); ok = false; break; }
       tc_fence_after();
       // the raw logits of this half row (rs > 0, so the maximum can be taken before scaling)
       float s[64];
@@ -406,7 +387,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           const float alpha = need ? exp2f(m_used - m_new) : 1.0f;     // 0 when nothing was unmasked so far
           if (need) m_used = m_new;
           l *= alpha;
-          if (!mbar_wait(&sm.pv_done[(j - 1) & 1][g], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
+          if (!mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
           tc_fence_after();
 #pragma unroll 1
           for (int c0 = 0; c0 < D; c0 += 32) {
@@ -420,33 +401,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           tmem_wait_st();
         }
       }
-      // P_g = 2^(S rs - m) as bf16 into row `row` of block g of P[sb], once the P V products of
-      // tile j-2 have consumed that buffer
-      if (j >= 2 && !mbar_wait(&sm.pv_done[sb][g], ((j >> 1) - 1) & 1)) { tf.raise(20); ok = false; break; }
+      // P_g = 2^(S rs - m) as bf16 pairs over the first 32 columns of this half row (which is in registers)
       const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
       float l4[4] = {0.f, 0.f, 0.f, 0.f};
-      unsigned char* prow = sm.p[sb] + g * kBlockBytes + (row >> 3) * 1024 + (row & 7) * 128;
+      uint32_t pk[32];
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {                 // 16-byte chunk ch = keys 8 ch .. 8 ch + 7 of this half
-        uint32_t w[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float p0 = exp2f(fmaf(s[ch * 8 + 2 * e], rs, neg_m));
-          const float p1 = exp2f(fmaf(s[ch * 8 + 2 * e + 1], rs, neg_m));
-          l4[e] += p0 + p1;
-          const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
-          w[e] = *reinterpret_cast<const uint32_t*>(&pp);
-        }
-        *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+      for (int c = 0; c < 32; ++c) {
+        const float p0 = exp2f(fmaf(s[2 * c], rs, neg_m));
+        const float p1 = exp2f(fmaf(s[2 * c + 1], rs, neg_m));
+        l4[c & 3] += p0 + p1;
+        const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
+        pk[c] = *reinterpret_cast<const uint32_t*>(&pp);
       }
+      tmem_st32(tmem + lane_base + colS, pk);
       l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
-      tc_fence_before();                               // this thread's TMEM loads (and rescale stores) are done
+      tmem_wait_st();
+      tc_fence_before();
       mbar_arrive(&sm.p_full[sb][g]);
     }
     // ---- epilogue: merge the two halves of the row, O / l -> bf16, row log2-sum-exp ----
-    if (ok && !(mbar_wait(&sm.pv_done[(nt - 1) & 1][0], ((nt - 1) >> 1) & 1) &&
-                mbar_wait(&sm.pv_done[(nt - 1) & 1][1], ((nt - 1) >> 1) & 1))) { tf.raise(19); ok = false; }
+    if (ok && !mbar_wait(&sm.pv_done[(nt - 1) & 1], ((nt - 1) >> 1) & 1)) { tf.raise(19); ok = false; }
     tc_fence_after();
     // the K ring is idle now (its last use completed before that P V product): exchange (max, sum) there
     float* xm = reinterpret_cast<float*>(sm.k[0]);    // [2][BT]
