@@ -172,6 +172,15 @@ int buzz_status(buzz_t ctx, void* stream);
 /* Number of kernels the library has launched through this object (for launch accounting). */
 int64_t buzz_launch_count(buzz_t ctx);
 
+/* Sampling variants of the paper's ablation study (Section 4.3). By default new tokens are sampled
+ * by local maximum with stride `segment` (Algorithm 2) and old tokens at intervals of
+ * s_hat = floor((segment+1)/2). This call replaces the two strides (e.g. swapped, the "small stride
+ * for old tokens" ablation) and, with interval_new != 0, samples new tokens at intervals as well
+ * (the "no local max" ablation: the first min(hitters, length) slots of every segment are kept and
+ * scores are ignored). Takes effect from the next prefill / eviction; counts stay score-independent.
+ * Rejects new_stride < 2, hitters >= new_stride, old_stride < 1, budget < sink + window + new_stride. */
+int buzz_set_sampling(buzz_t ctx, int interval_new, int new_stride, int old_stride);
+
 /* Tuning knob: number of CTAs (1, 2, 4 or 8) of the thread-block cluster that shares one instance's
  * slots in buzz_decode_step; 0 restores the built-in choice. Results do not depend on it beyond
  * fp32 summation order. */

@@ -45,6 +45,8 @@ struct Head {
   int g, d;
   int sink, window, segment, hitters, budget;
   int logn;            // 0: scale 1/sqrt(d) (Eq. 3); 1: scale log_512(n)/sqrt(d) (Section 3.5)
+  int old_stride = 0;  // stride for old tokens; 0 = the paper's s_hat = floor((s+1)/2)
+  int interval_new = 0;  // 1: interval sampling for new tokens too (the "no local max" ablation, Section 4.3)
   int n = 0, n_old = 0, total_len = 0;
   std::vector<double> K, V;   // [n][d], position order
   std::vector<double> score;  // [n]
@@ -74,7 +76,7 @@ int evict_once(Head& h) {
   const int k = h.sink, w = h.window, s = h.segment;
   if (h.n < h.budget) return 0;          // threshold buffering: evict only when full
   if (h.n <= k + w) return 0;            // Remark 1: sink and window are filled first
-  const int s_hat = (s + 1) / 2;         // floor((s+1)/2)
+  const int s_hat = h.old_stride > 0 ? h.old_stride : (s + 1) / 2;   // floor((s+1)/2) unless overridden (Section 4.3)
   const int new_begin = k + h.n_old;
   const int new_end = h.n - w;
 
@@ -87,6 +89,10 @@ int evict_once(Head& h) {
     const int hi = std::min(idx + s, new_end);
     const int want = std::min(h.hitters, hi - idx);
     std::vector<int> chosen;
+    if (h.interval_new) {                 // ablation: the first `want` slots of the hive, scores ignored
+      for (int r = 0; r < want; ++r) keep.push_back(idx + r);
+      continue;
+    }
     for (int r = 0; r < want; ++r) {
       int best = -1;
       for (int j = idx; j < hi; ++j) {
@@ -135,6 +141,18 @@ void* bo_create(int g, int d, int sink, int window, int segment, int hitters, in
 }
 
 void bo_destroy(void* p) { delete (Head*)p; }
+
+// Sampling variants of the ablation study (Section 4.3): interval sampling for new tokens as well,
+// and free choice of the two strides (e.g. swapped). new_stride replaces s, old_stride replaces s_hat.
+int bo_set_sampling(void* p, int interval_new, int new_stride, int old_stride) {
+  Head& h = *(Head*)p;
+  if (new_stride < 2 || h.hitters >= new_stride || old_stride < 1 || h.budget < h.sink + h.window + new_stride)
+    return BO_BAD_ARG;
+  h.segment = new_stride;
+  h.old_stride = old_stride;
+  h.interval_new = interval_new ? 1 : 0;
+  return BO_OK;
+}
 
 // Causal prefill (Eqs. 1 and 3) + initial scores + Remark 2's repeated sampling.
 //   Q [g][N][d], K [N][d], V [N][d] -> O [g][N][d]; full_score [N] (may be null) receives the

@@ -53,6 +53,8 @@ def _load():
         lib.bo_get_counts.argtypes = [ctypes.c_void_p, ip, ip, ip]
         lib.bo_get_state.argtypes = [ctypes.c_void_p, ip, dp, dp, dp]
         lib.bo_set_scores.argtypes = [ctypes.c_void_p, dp]
+        lib.bo_set_sampling.restype = c_int
+        lib.bo_set_sampling.argtypes = [ctypes.c_void_p, c_int, c_int, c_int]
         lib.bo_set_state.restype = c_int
         lib.bo_set_state.argtypes = [ctypes.c_void_p, c_int, c_int, c_int, ip, dp, dp, dp]
         _lib = lib
@@ -85,6 +87,13 @@ class OracleHead:
         if h:
             self._lib.bo_destroy(h)
             self._h = None
+
+    def set_sampling(self, interval_new, new_stride, old_stride):
+        """Ablation variants (Section 4.3): interval sampling for new tokens, free strides."""
+        rc = self._lib.bo_set_sampling(self._h, int(bool(interval_new)), int(new_stride), int(old_stride))
+        if rc < 0:
+            raise ValueError("oracle rejected the sampling parameters")
+        self.segment = int(new_stride)
 
     # -- the three steps -------------------------------------------------------------------
     def prefill(self, Q, K, V):

@@ -37,7 +37,7 @@ def exported_symbols() -> list[str]:
     return ["buzz_workspace_bytes", "buzz_create", "buzz_destroy", "buzz_prefill", "buzz_decode_step",
             "buzz_decode_step_host", "buzz_evict", "buzz_export_state", "buzz_import_state",
             "buzz_export_prefill_scores", "buzz_prefill_static",
-            "buzz_status", "buzz_launch_count", "buzz_set_decode_cluster", "buzz_error_string"]
+            "buzz_status", "buzz_launch_count", "buzz_set_decode_cluster", "buzz_set_sampling", "buzz_error_string"]
 
 
 def load_library(build_if_missing: bool = True):
@@ -78,6 +78,8 @@ def load_library(build_if_missing: bool = True):
     lib.buzz_status.argtypes = [vp, vp]
     lib.buzz_launch_count.restype = ctypes.c_int64
     lib.buzz_launch_count.argtypes = [vp]
+    lib.buzz_set_sampling.restype = ci
+    lib.buzz_set_sampling.argtypes = [vp, ci, ci, ci]
     lib.buzz_set_decode_cluster.restype = ci
     lib.buzz_set_decode_cluster.argtypes = [vp, ci]
     lib.buzz_error_string.restype = ctypes.c_char_p
@@ -179,6 +181,9 @@ class Buzz:
 
     def launch_count(self) -> int:
         return self._lib.buzz_launch_count(self._h)
+
+    def set_sampling(self, interval_new: bool, new_stride: int, old_stride: int):
+        _check(self._lib.buzz_set_sampling(self._h, int(bool(interval_new)), new_stride, old_stride), "buzz_set_sampling")
 
     def set_decode_cluster(self, cluster_size: int):
         _check(self._lib.buzz_set_decode_cluster(self._h, cluster_size), "buzz_set_decode_cluster")

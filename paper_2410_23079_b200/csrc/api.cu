@@ -91,7 +91,7 @@ int buzz_create(buzz_t* out, int sink, int window, int segment, int hitters, int
     return BUZZ_ERR_INVALID;
   buzz_ctx* c = new (std::nothrow) buzz_ctx();
   if (!c) return BUZZ_ERR_INVALID;
-  c->pol = BuzzPolicy{sink, window, segment, hitters, budget, (segment + 1) / 2};
+  c->pol = BuzzPolicy{sink, window, segment, hitters, budget, (segment + 1) / 2, 0};
   c->sh = *shape;
   c->group = shape->q_heads / shape->kv_heads;
   c->esize = shape->dtype == BUZZ_BF16 ? 2 : 4;
@@ -264,6 +264,17 @@ int buzz_status(buzz_t c, void* stream) {
 }
 
 int64_t buzz_launch_count(buzz_t c) { return c ? c->launches : 0; }
+
+int buzz_set_sampling(buzz_t c, int interval_new, int new_stride, int old_stride) {
+  if (!c) return BUZZ_ERR_INVALID;
+  if (new_stride < 2 || new_stride > 1024 || c->pol.hitters >= new_stride || old_stride < 1 ||
+      c->pol.budget < c->pol.sink + c->pol.window + new_stride)
+    return BUZZ_ERR_INVALID;
+  c->pol.segment = new_stride;
+  c->pol.s_hat = old_stride;
+  c->pol.interval_new = interval_new ? 1 : 0;
+  return BUZZ_OK;
+}
 
 int buzz_set_decode_cluster(buzz_t c, int cluster_size) {
   if (!c) return BUZZ_ERR_INVALID;

@@ -15,7 +15,8 @@ struct BuzzPolicy {
   int segment;   // s
   int hitters;   // winners per segment
   int budget;    // T + k + w
-  int s_hat;     // floor((s+1)/2)
+  int s_hat;     // stride for old tokens: floor((s+1)/2) unless overridden
+  int interval_new;  // 1: interval sampling for new tokens too (ablation), 0: local max (Algorithm 2)
 };
 
 // Device view of the persistent state. Instance index = ((layer * max_batch) + seq) * kv_heads + head.

@@ -69,6 +69,10 @@ evict_kernel(BuzzState st, BuzzPolicy pol, int layer_begin, int max_batch, int k
     const int len = min(s, new_end - lo);
     const int want = min(h, len);
     const int out0 = pol.sink + kept_old + seg * h;
+    if (pol.interval_new) {                         // ablation: the first `want` slots of the segment
+      for (int r = lane; r < want; r += 32) src[out0 + r] = lo + r;
+      continue;
+    }
     unsigned chosen = 0;                            // bit i: candidate lo + i*32 + lane is a winner
     for (int r = 0; r < want; ++r) {
       Cand best{0.f, -1};

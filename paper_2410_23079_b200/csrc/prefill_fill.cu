@@ -48,6 +48,7 @@ __device__ inline int round_one_winner(const float* __restrict__ sc, int N, cons
   const int lo = pol.sink + seg * pol.segment;
   const int hi = min(lo + pol.segment, N - pol.window);
   const int want = min(pol.hitters, hi - lo);
+  if (pol.interval_new) return lo + rank;           // ablation: interval sampling, scores ignored
   if (want == 1) {
     int best = lo;
     float bv = sc[lo];

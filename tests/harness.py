@@ -90,7 +90,8 @@ def check_prefill_sampled(w, Q, K, V, got, gpu_scores, rows, tail_keys, tol, log
 
 
 def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None, check_every=1,
-                 device="cuda:0", logn=False, bz: Buzz | None = None, sampled_rows=None, tail_keys=64):
+                 device="cuda:0", logn=False, bz: Buzz | None = None, sampled_rows=None, tail_keys=64,
+                 sampling=None):
     """Runs prefill + decode/evict on the GPU for the whole workload and the oracle on `samples`
     (a list of (layer, seq, kv_head)). Returns a dict of summary counters."""
     tol = TOL[w.dtype]
@@ -98,6 +99,8 @@ def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None,
     layers = list(range(w.layers)) if layers is None else layers
     own = bz is None
     bz = bz or make_buzz(w, device, logn=logn)
+    if sampling is not None:                     # (interval_new, new_stride, old_stride): Section 4.3 variants
+        bz.set_sampling(*sampling)
     lens = workloads.prompt_lengths(w)
     offs = np.concatenate([[0], np.cumsum(lens)])
     g, d = w.group, w.head_dim
@@ -123,6 +126,8 @@ def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None,
             gs = pscore[h][a:e]
             if sampled_rows is None:
                 free = OracleHead(g, d, w.sink, w.window, w.segment, w.hitters, w.budget, logn=logn)
+                if sampling is not None:
+                    free.set_sampling(*sampling)
                 O, full, rounds = free.prefill(Q, K, V)
                 stats["prefill_rounds"] = max(stats["prefill_rounds"], rounds)
                 assert_close(got, O, what=f"prefill out L{layer} b{b} h{h}", **tol)
@@ -133,6 +138,8 @@ def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None,
                                       f"L{layer} b{b} h{h}", stats)
             # lock-step instance: selection decided on the GPU's fp32 scores
             ls = OracleHead(g, d, w.sink, w.window, w.segment, w.hitters, w.budget, logn=logn)
+            if sampling is not None:
+                ls.set_sampling(*sampling)
             N = e - a
             ls.set_state(0, N, np.arange(N), gs.astype(np.float64), K, V)
             while ls.counts()[0] >= w.budget:

@@ -251,3 +251,24 @@ def test_prefill_is_reproducible_at_full_size(cuda_device):
             assert torch.equal(sc, ref_sc)
             assert torch.equal(st["pos"], ref_st["pos"]) and torch.equal(st["score"], ref_st["score"])
     bz.close()
+
+
+@pytest.mark.parametrize("sampling", [(False, 4, 8), (True, 8, 4), (True, 5, 3)])
+def test_sampling_variants_of_the_ablation_study(cuda_device, sampling):
+    """Section 4.3 variants (swapped strides; interval sampling for new tokens) through prefill-time
+    rounds and decode-time evictions, lock-step against the oracle."""
+    w = workloads.scaled(workloads.get("C2"), layers=2, batch=2, q_heads=2, kv_heads=2, prompt_min=650,
+                         prompt_max=650, decode_steps=120, window=48, budget=150, hitters=1)
+    stats = run_lockstep(w, [(0, 0, 0), (1, 1, 1)], check_every=7, sampling=sampling)
+    assert stats["evictions"] >= 2
+
+
+def test_sampling_variant_validation(cuda_device):
+    from paper_2410_23079_b200 import BuzzError
+    w = workloads.scaled(workloads.get("C1"), hitters=3, segment=8, budget=120)
+    bz = make_buzz(w, max_prompt_tokens=64)
+    for bad in [(False, 1, 2), (False, 3, 2), (False, 8, 0), (False, 60, 2)]:
+        with pytest.raises(BuzzError):
+            bz.set_sampling(*bad)
+    bz.set_sampling(True, 8, 4)
+    bz.close()

@@ -199,3 +199,54 @@ def test_parameter_validation():
         p.update(bad)
         with pytest.raises(ValueError):
             OracleHead(1, 4, **p)
+
+
+def _interval_reference(lo, hi, s, hmax):
+    out = []
+    for a in range(lo, hi, s):
+        out += list(range(a, min(a + min(hmax, s), hi)))
+    return out
+
+
+@pytest.mark.parametrize("interval_new,new_stride,old_stride", [(False, 3, 5), (True, 6, 3), (True, 4, 1), (False, 7, 2)])
+def test_sampling_variants_of_the_ablation_study(interval_new, new_stride, old_stride):
+    """Section 4.3: swapped / free strides and interval sampling for new tokens, against a selection
+    written independently here; counts follow a_n = ceil(a/s_old) + kept(T - a) whatever the scores."""
+    rng = np.random.default_rng(new_stride * 10 + old_stride)
+    sink, window, hit, T = 3, 11, 2 if new_stride > 2 else 1, 90
+    budget = sink + window + T
+    h = OracleHead(1, 1, sink, window, 16, hit, budget)
+    h.set_sampling(interval_new, new_stride, old_stride)
+    n0 = sink + window
+    h.set_state(0, n0, np.arange(n0), rng.random(n0), np.zeros((n0, 1)), np.zeros((n0, 1)))
+    evictions = 0
+    for t in range(n0, n0 + 600):
+        h.decode(np.zeros((1, 1)), np.zeros(1), np.zeros(1))
+        n, n_old, _ = h.counts()
+        sc = np.round(rng.random(n) * 5) / 5
+        h.set_scores(sc)
+        pos, _ = h.state(with_kv=False)
+        r = h.evict()
+        if n < budget:
+            assert r == 0
+            continue
+        old_keep = list(range(sink, sink + n_old, old_stride))
+        lo, hi = sink + n_old, n - window
+        new_keep = _interval_reference(lo, hi, new_stride, hit) if interval_new else \
+            _segment_winners_reference(sc, lo, hi, new_stride, hit)
+        expect = list(range(sink)) + old_keep + new_keep + list(range(n - window, n))
+        if len(expect) >= n:                      # nothing can be dropped (old stride 1): reported, not looped
+            assert r == BO_NO_PROGRESS
+            break
+        assert r == 1
+        evictions += 1
+        assert h.state(with_kv=False)[0].tolist() == pos[expect].tolist()
+        assert h.counts()[1] == len(old_keep) + len(new_keep)
+    assert evictions >= 3 or old_stride == 1
+
+
+def test_sampling_variant_validation():
+    h = OracleHead(1, 1, 2, 4, 8, 3, 40)
+    for bad in [(False, 1, 2), (False, 3, 2), (False, 8, 0), (False, 40, 2)]:
+        with pytest.raises(ValueError):
+            h.set_sampling(*bad)
