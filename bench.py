@@ -265,18 +265,22 @@ def run_ours(args):
 
     # ---- end-to-end leg: the same step through the host-buffer entry point -------------------
     Ke = min(K, args.e2e_steps)
-    hq = [torch.empty((pool,) + tuple(dec[l][0].shape[1:]), dtype=dt).pin_memory() for l in range(w.layers)]
-    hk = [torch.empty((pool,) + tuple(dec[l][1].shape[1:]), dtype=dt).pin_memory() for l in range(w.layers)]
-    hv = [torch.empty((pool,) + tuple(dec[l][2].shape[1:]), dtype=dt).pin_memory() for l in range(w.layers)]
+    # pinned host inputs, one packed q|k|v record per (layer, step) so that a step's inputs go down in one copy
+    nq = w.batch * w.q_heads * w.head_dim
+    nk = w.batch * w.kv_heads * w.head_dim
+    hin = [torch.empty((pool, nq + 2 * nk), dtype=dt).pin_memory() for l in range(w.layers)]
     ho = [torch.empty(tuple(dec[l][0].shape[1:]), dtype=dt).pin_memory() for l in range(w.layers)]
     for l in range(w.layers):
-        hq[l].copy_(dec[l][0]); hk[l].copy_(dec[l][1]); hv[l].copy_(dec[l][2])
+        hin[l][:, :nq].copy_(dec[l][0].reshape(pool, nq))
+        hin[l][:, nq:nq + nk].copy_(dec[l][1].reshape(pool, nk))
+        hin[l][:, nq + nk:].copy_(dec[l][2].reshape(pool, nk))
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for i in range(Ke):
         for layer in range(w.layers):
-            bz.decode_step_host(layer, hq[layer][t % pool], hk[layer][t % pool], hv[layer][t % pool], ho[layer])
+            rec = hin[layer][t % pool]
+            bz.decode_step_host(layer, rec[:nq], rec[nq:nq + nk], rec[nq + nk:], ho[layer])
         bz.evict(-1)
         advance_counts(); t += 1
     e1.record(stream)

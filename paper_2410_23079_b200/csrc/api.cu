@@ -169,13 +169,20 @@ int buzz_decode_step_host(buzz_t c, int layer, const void* q_host, const void* k
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t qb = (size_t)batch * c->sh.q_heads * c->sh.head_dim * c->esize;
   const size_t kb = (size_t)batch * c->sh.kv_heads * c->sh.head_dim * c->esize;
+  // staging is packed q | k | v (row sizes are multiples of 16 bytes), so host buffers laid out the
+  // same way go down in ONE copy; `out` has its own region behind them
   char* dq = c->stage;
-  char* dk = dq + c->stage_q;
-  char* dv = dk + c->stage_kv;
-  char* dout = dv + c->stage_kv;
-  if (cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
-  if (cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
-  if (cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+  char* dk = dq + qb;
+  char* dv = dk + kb;
+  char* dout = c->stage + c->stage_q + 2 * c->stage_kv;
+  const char* qh = static_cast<const char*>(q_host);
+  if (static_cast<const char*>(k_new_host) == qh + qb && static_cast<const char*>(v_new_host) == qh + qb + kb) {
+    if (cudaMemcpyAsync(dq, q_host, qb + 2 * kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+  } else {
+    if (cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+  }
   if (buzz_launch_decode(c, layer, dq, dk, dv, dout, s) != cudaSuccess) return BUZZ_ERR_CUDA;
   if (cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return BUZZ_ERR_CUDA;
   return BUZZ_OK;

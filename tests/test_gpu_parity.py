@@ -272,3 +272,34 @@ def test_sampling_variant_validation(cuda_device):
             bz.set_sampling(*bad)
     bz.set_sampling(True, 8, 4)
     bz.close()
+
+
+def test_decode_step_host_matches_device_entry(cuda_device):
+    """The host-buffer entry point (separate and packed q|k|v records) gives bit-identical outputs and
+    caches to the device-pointer entry point."""
+    w = workloads.scaled(workloads.get("C4"), layers=1, batch=2, q_heads=8, kv_heads=2, prompt_min=260,
+                         prompt_max=260, decode_steps=6, window=32, budget=300)
+    q, k, v, cu = workloads.prefill_inputs(w, 0, "cuda:0")
+    qd, kd, vd = workloads.decode_inputs(w, 0, "cuda:0")
+    ref, sep, packed = make_buzz(w), make_buzz(w), make_buzz(w)
+    for bz in (ref, sep, packed):
+        bz.prefill(0, q, k, v, cu, 260, torch.empty_like(q))
+    nq, nk = qd[0].numel(), kd[0].numel()
+    for t in range(w.decode_steps):
+        o_ref = torch.empty_like(qd[t])
+        ref.decode_step(0, qd[t], kd[t], vd[t], o_ref)
+        hq, hk, hv = qd[t].cpu().pin_memory(), kd[t].cpu().pin_memory(), vd[t].cpu().pin_memory()
+        o_sep = torch.empty_like(hq).pin_memory()
+        sep.decode_step_host(0, hq, hk, hv, o_sep)
+        rec = torch.cat([hq.reshape(-1), hk.reshape(-1), hv.reshape(-1)]).pin_memory()
+        o_pk = torch.empty_like(hq).pin_memory()
+        packed.decode_step_host(0, rec[:nq], rec[nq:nq + nk], rec[nq + nk:], o_pk)
+        torch.cuda.synchronize()
+        assert torch.equal(o_sep, o_ref.cpu()) and torch.equal(o_pk, o_ref.cpu())
+    for bz in (sep, packed):
+        for b in range(2):
+            a, c = ref.export_state(0, b, 1), bz.export_state(0, b, 1)
+            assert a["n"] == c["n"] and torch.equal(a["score"], c["score"]) and torch.equal(a["k"], c["k"])
+        assert bz.status() == 0
+    for bz in (ref, sep, packed):
+        bz.close()
