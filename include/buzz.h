@@ -132,7 +132,8 @@ int buzz_decode_step(buzz_t ctx, int layer, const void* q, const void* k_new, co
 /* The same step with HOST buffers (pinned memory recommended): copies q/k_new/v_new to the
  * library's staging area in scratch, runs the step, copies `out` back, all on `stream`, without
  * synchronising. Layouts as in buzz_decode_step. If the three inputs are contiguous in host memory in
- * the order q, k_new, v_new they are sent in a single copy. */
+ * the order q, k_new, v_new (one allocation holding the packed record) they are sent in a single
+ * copy; buffers that merely happen to be adjacent but were pinned separately are copied one by one. */
 int buzz_decode_step_host(buzz_t ctx, int layer, const void* q_host, const void* k_new_host,
                           const void* v_new_host, void* out_host, void* stream);
 

@@ -176,9 +176,14 @@ int buzz_decode_step_host(buzz_t c, int layer, const void* q_host, const void* k
   char* dv = dk + kb;
   char* dout = c->stage + c->stage_q + 2 * c->stage_kv;
   const char* qh = static_cast<const char*>(q_host);
+  bool sent = false;
   if (static_cast<const char*>(k_new_host) == qh + qb && static_cast<const char*>(v_new_host) == qh + qb + kb) {
-    if (cudaMemcpyAsync(dq, q_host, qb + 2 * kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
-  } else {
+    // Adjacent addresses do not prove one allocation: a copy that spans separately pinned buffers is
+    // refused at the call ("invalid argument", nothing queued). Then clear that error and copy by parts.
+    sent = cudaMemcpyAsync(dq, q_host, qb + 2 * kb, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (!sent) (void)cudaGetLastError();
+  }
+  if (!sent) {
     if (cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
     if (cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
     if (cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;

@@ -154,6 +154,7 @@ cudaError_t buzz_launch_evict(buzz_ctx* c, int layer_begin, int layer_count, cud
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) batch = max(batch, c->batch[l]);
   if (batch == 0) return cudaSuccess;
   dim3 grid(c->sh.kv_heads, batch, layer_count);
+  (void)cudaGetLastError();   // drop a stale non-sticky error left by an earlier runtime call of the process
   const size_t smem = (size_t)c->pol.budget * sizeof(int32_t);
   const int row_bytes = c->sh.head_dim * (int)c->esize;
 #define BUZZ_EVICT_CASE(RB)                                                                        \

@@ -128,6 +128,7 @@ cudaError_t buzz_launch_prefill_fill(buzz_ctx* c, int layer, const void* k, cons
   int bx = (n_max + slots - 1) / slots;
   if (bx < 1) bx = 1;
   dim3 grid(bx, c->sh.kv_heads, batch);
+  (void)cudaGetLastError();   // drop a stale non-sticky error left by an earlier runtime call of the process
 #define BUZZ_FILL_CASE(RB)                                                                      \
   case RB:                                                                                      \
     prefill_fill_kernel<RB><<<grid, kThreads, 0, stream>>>(                                     \

@@ -228,6 +228,7 @@ cudaError_t launch_simt(buzz_ctx* c, const void* q, const void* k, const void* v
   const int tiles = (max_seqlen + BM - 1) / BM;
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
   const int logn = (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0;
+  (void)cudaGetLastError();   // drop a stale non-sticky error left by an earlier runtime call of the process
   prefill_attn_kernel<T, D><<<dim3(tiles, c->sh.q_heads, batch), kThreads, smemA, stream>>>(
       (const T*)q, (const T*)k, (const T*)v, cu, (T*)out, c->lse, c->sh.q_heads, c->sh.kv_heads,
       c->sh.max_prompt_tokens, scale_log2, logn);

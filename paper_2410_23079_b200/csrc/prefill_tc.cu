@@ -520,6 +520,7 @@ cudaError_t buzz_launch_prefill_tc(buzz_ctx* c, const void* q, const void* k, co
   const int tiles = (max_seqlen + BT - 1) / BT;
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
   const int logn = (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0;
+  (void)cudaGetLastError();   // drop a stale non-sticky error left by an earlier runtime call of the process
   attn_tc_kernel<<<dim3(tiles, c->sh.q_heads, batch), kThreadsA, smemA, stream>>>(
       mq, mk, mv, cu, (__nv_bfloat16*)out, c->lse, c->st.status, c->sh.q_heads, c->sh.kv_heads,
       c->sh.max_prompt_tokens, scale_log2, logn);
