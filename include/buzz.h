@@ -66,7 +66,7 @@ enum {
  *   state   : K and V caches [L][max_batch][Hkv][budget][d], score and pos [L][max_batch][Hkv][budget],
  *             counters n / n_old / total_len [L][max_batch][Hkv], and the status words.
  *   scratch : per-row softmax statistics and per-key column sums of one prefill, plus staging
- *             buffers for buzz_decode_step_host. Contents are not carried between calls.
+ *             buffers (one set per layer) for the host-buffer decode entries. Contents are not carried between calls.
  * Returns BUZZ_ERR_INVALID for a shape or budget the library does not support. */
 int buzz_workspace_bytes(const buzz_shape* shape, int budget, size_t* state_bytes, size_t* scratch_bytes);
 
@@ -136,6 +136,29 @@ int buzz_decode_step(buzz_t ctx, int layer, const void* q, const void* k_new, co
  * copy; buffers that merely happen to be adjacent but were pinned separately are copied one by one. */
 int buzz_decode_step_host(buzz_t ctx, int layer, const void* q_host, const void* k_new_host,
                           const void* v_new_host, void* out_host, void* stream);
+
+/* One decode step (Eqs. 2 and 3) of SEVERAL layers in one call: the attention-only step of a layer
+ * stack whose per-layer inputs already exist, e.g. a benchmark of the cache policy or a caller
+ * that batches independent attention calls. `layers` (host array of `count` pairwise distinct
+ * layer indices) is walked in order; q, k_new, v_new and out are host arrays of `count` device
+ * pointers with the layouts of buzz_decode_step for each layer's own batch. Results are those of
+ * `count` buzz_decode_step calls.
+ * Contract: every input buffer must be complete (in stream order) before this call, and no `out`
+ * buffer may alias another member's buffers. Within the call the launches are NOT serialised:
+ * CTAs of consecutive layers occupy the SMs back to back and each member finishes only after the
+ * members before it, so work enqueued after the call sees all of them complete. The first member
+ * waits for all earlier work in the stream.
+ * Returns BUZZ_ERR_INVALID for a repeated or out-of-range layer or a null / misaligned pointer. */
+int buzz_decode_layers(buzz_t ctx, int count, const int* layers, const void* const* q,
+                       const void* const* k_new, const void* const* v_new, void* const* out,
+                       void* stream);
+
+/* buzz_decode_layers with HOST buffers (pinned memory recommended). `in_host` is one packed buffer,
+ * for each listed layer in order its q | k_new | v_new tensors (layouts of buzz_decode_step, sized by
+ * that layer's batch); `out_host` receives the outputs packed the same way. One host-to-device
+ * copy, the launches, one device-to-host copy, all on `stream`, without synchronising. */
+int buzz_decode_layers_host(buzz_t ctx, int count, const int* layers, const void* in_host,
+                            void* out_host, void* stream);
 
 /* BUZZ eviction (Algorithm 1's sampling line and final concatenation; Algorithm 2) for one layer,
  * or for all layers when layer = -1. Per instance, entirely on the device: nothing happens unless

@@ -35,7 +35,7 @@ class _Shape(ctypes.Structure):
 def exported_symbols() -> list[str]:
     """Every entry point include/buzz.h declares."""
     return ["buzz_workspace_bytes", "buzz_create", "buzz_destroy", "buzz_prefill", "buzz_decode_step",
-            "buzz_decode_step_host", "buzz_evict", "buzz_export_state", "buzz_import_state",
+            "buzz_decode_step_host", "buzz_decode_layers", "buzz_decode_layers_host", "buzz_evict", "buzz_export_state", "buzz_import_state",
             "buzz_export_prefill_scores", "buzz_prefill_static",
             "buzz_status", "buzz_launch_count", "buzz_set_decode_cluster", "buzz_set_sampling", "buzz_error_string"]
 
@@ -66,6 +66,10 @@ def load_library(build_if_missing: bool = True):
     lib.buzz_decode_step.argtypes = [vp, ci, vp, vp, vp, vp, vp]
     lib.buzz_decode_step_host.restype = ci
     lib.buzz_decode_step_host.argtypes = [vp, ci, vp, vp, vp, vp, vp]
+    lib.buzz_decode_layers.restype = ci
+    lib.buzz_decode_layers.argtypes = [vp, ci, ctypes.POINTER(ci)] + [ctypes.POINTER(vp)] * 4 + [vp]
+    lib.buzz_decode_layers_host.restype = ci
+    lib.buzz_decode_layers_host.argtypes = [vp, ci, ctypes.POINTER(ci), vp, vp, vp]
     lib.buzz_evict.restype = ci
     lib.buzz_evict.argtypes = [vp, ci, vp]
     lib.buzz_export_state.restype = ci
@@ -171,6 +175,23 @@ class Buzz:
         _check(self._lib.buzz_decode_step_host(self._h, layer, q.data_ptr(), k_new.data_ptr(),
                                                v_new.data_ptr(), out.data_ptr(), _stream_ptr(stream)),
                "buzz_decode_step_host")
+
+    def decode_layers(self, layers, q, k_new, v_new, out, stream=None):
+        """buzz_decode_layers: one decode step of several distinct layers whose inputs (lists of device
+        tensors, one per layer) are all complete; the launches overlap on the GPU."""
+        n = len(layers)
+        ci, vp = ctypes.c_int, ctypes.c_void_p
+        arr = lambda ts: (vp * n)(*[t.data_ptr() for t in ts])
+        _check(self._lib.buzz_decode_layers(self._h, n, (ci * n)(*layers), arr(q), arr(k_new), arr(v_new),
+                                            arr(out), _stream_ptr(stream)), "buzz_decode_layers")
+
+    def decode_layers_host(self, layers, in_host, out_host, stream=None):
+        """buzz_decode_layers_host: `in_host` holds, per listed layer, q | k_new | v_new packed back to
+        back; `out_host` receives the outputs packed in the same order."""
+        n = len(layers)
+        _check(self._lib.buzz_decode_layers_host(self._h, n, (ctypes.c_int * n)(*layers), in_host.data_ptr(),
+                                                 out_host.data_ptr(), _stream_ptr(stream)),
+               "buzz_decode_layers_host")
 
     def evict(self, layer=-1, stream=None):
         _check(self._lib.buzz_evict(self._h, layer, _stream_ptr(stream)), "buzz_evict")

@@ -56,7 +56,7 @@ Layout make_layout(const buzz_shape& s, int budget) {
   L.pscore = off; off = align_up(off + (size_t)s.kv_heads * s.max_prompt_tokens * sizeof(float));
   L.stage_q = align_up((size_t)s.max_batch * s.q_heads * s.head_dim * e);
   L.stage_kv = align_up((size_t)s.max_batch * s.kv_heads * s.head_dim * e);
-  L.stage = off; off += 2 * L.stage_q + 2 * L.stage_kv;
+  L.stage = off; off += (size_t)s.layers * (2 * L.stage_q + 2 * L.stage_kv);
   L.scratch_bytes = off;
   return L;
 }
@@ -174,7 +174,7 @@ int buzz_decode_step_host(buzz_t c, int layer, const void* q_host, const void* k
   char* dq = c->stage;
   char* dk = dq + qb;
   char* dv = dk + kb;
-  char* dout = c->stage + c->stage_q + 2 * c->stage_kv;
+  char* dout = c->stage + (size_t)c->sh.layers * (c->stage_q + 2 * c->stage_kv);
   const char* qh = static_cast<const char*>(q_host);
   bool sent = false;
   if (static_cast<const char*>(k_new_host) == qh + qb && static_cast<const char*>(v_new_host) == qh + qb + kb) {
@@ -190,6 +190,75 @@ int buzz_decode_step_host(buzz_t c, int layer, const void* q_host, const void* k
   }
   if (buzz_launch_decode(c, layer, dq, dk, dv, dout, s) != cudaSuccess) return BUZZ_ERR_CUDA;
   if (cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+  return BUZZ_OK;
+}
+
+namespace {
+// layers of one multi-layer call: in range, prefilled or empty, and pairwise distinct
+bool layers_ok(buzz_t c, int count, const int* layers) {
+  if (!c || !layers || count < 1 || count > c->sh.layers) return false;
+  for (int i = 0; i < count; ++i) {
+    if (layers[i] < 0 || layers[i] >= c->sh.layers) return false;
+    for (int j = 0; j < i; ++j)
+      if (layers[j] == layers[i]) return false;
+  }
+  return true;
+}
+}  // namespace
+
+int buzz_decode_layers(buzz_t c, int count, const int* layers, const void* const* q,
+                       const void* const* k_new, const void* const* v_new, void* const* out,
+                       void* stream) {
+  if (!layers_ok(c, count, layers) || !q || !k_new || !v_new || !out) return BUZZ_ERR_INVALID;
+  for (int i = 0; i < count; ++i) {
+    if (!q[i] || !k_new[i] || !v_new[i] || !out[i]) return BUZZ_ERR_INVALID;
+    if (!aligned16(q[i]) || !aligned16(k_new[i]) || !aligned16(v_new[i]) || !aligned16(out[i])) return BUZZ_ERR_INVALID;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int pos = 0;                 // launches made so far in this call (empty layers launch nothing)
+  for (int i = 0; i < count; ++i) {
+    if (c->batch[layers[i]] == 0) continue;
+    int next = -1;
+    for (int j = i + 1; j < count && next < 0; ++j)
+      if (c->batch[layers[j]] != 0) next = layers[j];
+    if (buzz_launch_decode(c, layers[i], q[i], k_new[i], v_new[i], out[i], s, pos, next) != cudaSuccess)
+      return BUZZ_ERR_CUDA;
+    ++pos;
+  }
+  return BUZZ_OK;
+}
+
+int buzz_decode_layers_host(buzz_t c, int count, const int* layers, const void* in_host, void* out_host,
+                            void* stream) {
+  if (!layers_ok(c, count, layers) || !in_host || !out_host) return BUZZ_ERR_INVALID;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t row_q = (size_t)c->sh.q_heads * c->sh.head_dim * c->esize;
+  const size_t row_kv = (size_t)c->sh.kv_heads * c->sh.head_dim * c->esize;
+  size_t in_bytes = 0, out_bytes = 0;
+  for (int i = 0; i < count; ++i) {
+    in_bytes += c->batch[layers[i]] * (row_q + 2 * row_kv);
+    out_bytes += c->batch[layers[i]] * row_q;
+  }
+  if (in_bytes == 0) return BUZZ_OK;
+  char* din = c->stage;
+  char* dout = c->stage + (size_t)c->sh.layers * (c->stage_q + 2 * c->stage_kv);
+  if (cudaMemcpyAsync(din, in_host, in_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+  size_t io = 0, oo = 0;
+  int pos = 0;
+  for (int i = 0; i < count; ++i) {
+    const size_t b = c->batch[layers[i]];
+    if (b == 0) continue;
+    int next = -1;
+    for (int j = i + 1; j < count && next < 0; ++j)
+      if (c->batch[layers[j]] != 0) next = layers[j];
+    const char* dq = din + io;
+    if (buzz_launch_decode(c, layers[i], dq, dq + b * row_q, dq + b * (row_q + row_kv), dout + oo, s, pos, next) != cudaSuccess)
+      return BUZZ_ERR_CUDA;
+    io += b * (row_q + 2 * row_kv);
+    oo += b * row_q;
+    ++pos;
+  }
+  if (cudaMemcpyAsync(out_host, dout, out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return BUZZ_ERR_CUDA;
   return BUZZ_OK;
 }
 

@@ -40,7 +40,7 @@ struct buzz_ctx {
   // scratch partition
   float* lse;         // [q_heads][max_prompt_tokens] row log-sum-exp (log2 domain) of one prefill
   float* pscore;      // [kv_heads][max_prompt_tokens] pre-eviction prompt scores
-  char* stage;        // staging for buzz_decode_step_host: q | k | v | out
+  char* stage;        // staging for the host-buffer entries: per layer q | k | v, then per layer out
   size_t stage_q, stage_kv;  // byte sizes of one q-shaped and one kv-shaped staging tensor
   int* batch;         // active sequences per layer (host array)
   int decode_cluster; // 0 = choose automatically
@@ -63,8 +63,12 @@ __device__ inline void buzz_set_status(int32_t* status, int code, int inst, int 
 }
 
 // ---- launch wrappers (each returns a cudaError_t from the launch) ---------------------------
+// chain_pos: -1 for a single-layer call, else the index of this launch within one multi-layer call
+// (whose inputs are all complete before the call and whose layers are distinct); next_layer: the
+// layer the following launch will read (-1 unknown), used only as a prefetch hint.
 cudaError_t buzz_launch_decode(buzz_ctx* c, int layer, const void* q, const void* k_new,
-                               const void* v_new, void* out, cudaStream_t stream);
+                               const void* v_new, void* out, cudaStream_t stream, int chain_pos = -1,
+                               int next_layer = -1);
 cudaError_t buzz_launch_evict(buzz_ctx* c, int layer_begin, int layer_count, cudaStream_t stream);
 cudaError_t buzz_launch_prefill_attention(buzz_ctx* c, const void* q, const void* k, const void* v,
                                           const int32_t* cu, int batch, int total_tokens,

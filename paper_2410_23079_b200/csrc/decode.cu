@@ -332,10 +332,12 @@ cudaError_t launch_g(buzz_ctx* c, int layer, const void* q, const void* k_new, c
 }  // namespace
 
 cudaError_t buzz_launch_decode_bf16(buzz_ctx* c, int layer, const void* q, const void* k_new,
-                                    const void* v_new, void* out, int cluster_size, int early, cudaStream_t stream);
+                                    const void* v_new, void* out, int cluster_size, int mode, int next_layer,
+                                    cudaStream_t stream);
 
 cudaError_t buzz_launch_decode(buzz_ctx* c, int layer, const void* q, const void* k_new,
-                               const void* v_new, void* out, cudaStream_t stream) {
+                               const void* v_new, void* out, cudaStream_t stream, int chain_pos,
+                               int next_layer) {
   if (c->batch[layer] == 0) return cudaSuccess;
   int cs = c->decode_cluster;
   if (cs == 0) {
@@ -350,10 +352,14 @@ cudaError_t buzz_launch_decode(buzz_ctx* c, int layer, const void* q, const void
   while (cs < kMaxCluster && (size_t)c->group * ((c->pol.budget + cs - 1) / cs) * sizeof(float) > 96 * 1024) cs *= 2;
   cudaError_t e;
   if (c->sh.dtype == BUZZ_BF16) {
-    // the kernel may start reading this layer's cache while the previous launch drains only if that
-    // launch was a decode step of another layer issued through this object on the same stream
-    const int early = (c->last_kind == 1 && c->last_layer != layer && c->last_stream == (void*)stream) ? 1 : 0;
-    e = buzz_launch_decode_bf16(c, layer, q, k_new, v_new, out, cs, early, stream);   // tensor-core kernel
+    // Dependency mode of the kernel (see decode_bf16.cu). A later member of one multi-layer call
+    // overlaps with the members before it; a single call may only warm L2 ahead of its wait, and
+    // only if the launch before it was a decode step of another layer through this object and stream.
+    int mode = 0;
+    if (chain_pos > 0) mode = 2;
+    else if (chain_pos < 0 && c->last_kind == 1 && c->last_layer != layer && c->last_stream == (void*)stream) mode = 1;
+    if (chain_pos < 0) next_layer = layer + 1 == c->sh.layers ? 0 : layer + 1;   // a layer stack is walked in order
+    e = buzz_launch_decode_bf16(c, layer, q, k_new, v_new, out, cs, mode, next_layer, stream);   // tensor-core kernel
     if (e == cudaSuccess) { c->last_kind = 1; c->last_layer = layer; c->last_stream = (void*)stream; }
   } else {
     e = c->sh.head_dim == 128 ? launch_g<float, 128>(c, layer, q, k_new, v_new, out, cs, stream)

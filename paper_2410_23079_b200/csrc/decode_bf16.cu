@@ -33,6 +33,11 @@ constexpr int kMaxCluster = 8;
 constexpr int kHeads = 8;       // MMA column count: query heads of one group, zero-padded
 constexpr int kTile = 16;       // keys per warp tile
 constexpr int kPrefetchLines = 256;   // 128-byte lines of K a CTA may pull towards L2 before its wait (measured best)
+#ifndef BUZZ_DECODE_PD
+#define BUZZ_DECODE_PD 2
+#endif
+enum { kWaitFirst = 0, kHintFirst = 1, kOverlap = 2 };
+constexpr int kAhead = BUZZ_DECODE_PD;   // rolling L2 prefetch distance, in loop iterations (kWarps * kTile rows each)
 
 __device__ inline uint4 ld_stream(const uint4* p) { return __ldcs(p); }
 
@@ -65,7 +70,7 @@ __global__ void __launch_bounds__(kThreads)
 decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict__ q,
                    const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
                    __nv_bfloat16* __restrict__ out, int layer, int max_batch, int kv_heads,
-                   int chunk_cap, float scale_log2, int logn, int early) {
+                   int chunk_cap, float scale_log2, int logn, int mode, int next_layer) {
   constexpr int NCH = D / 8;          // 16-byte chunks per row
   constexpr int KL = NCH / 4;         // K chunks per lane and row
   constexpr int VJ = NCH / 8;         // V chunks per lane and row
@@ -89,15 +94,29 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   float* owarp = invL + G;                                   // [kWarps][G][D]
   float* sl = owarp + kWarps * G * D;                        // [G][chunk_cap] logits (log2 domain)
 
-  // Programmatic dependent launch. `early` is set by the host only when the kernel launched just
-  // before this one through the same object and stream was a decode step of ANOTHER layer: nothing
-  // it writes is read here before the wait, so this kernel may read its own layer's counters and
-  // pull the head of its K rows towards L2 while that kernel drains. Otherwise it waits first.
-  // A kernel triggers its dependents only where its own pre-wait reads are safe to begin.
-  if (early) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  else {
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // Programmatic dependent launch; the host picks one of three modes.
+  //   kWaitFirst  wait for everything earlier in the stream, then let the next launch begin.
+  //   kHintFirst  the launch just before this one (same object, same stream) was a decode step of
+  //               another layer: let the next launch begin, pull the head of this chunk's K rows
+  //               towards L2 using a possibly stale length, then wait, then read everything for real.
+  //   kOverlap    this launch is a later member of one buzz_decode_layers call: all inputs of the
+  //               call were complete before its first kernel (a kWaitFirst one) passed its wait, and
+  //               no other member touches this layer, so the whole step runs without waiting and
+  //               CTAs of consecutive layers fill the SMs back to back. The wait moves to the end
+  //               (before `out` is written), which keeps completion in stream order.
+  if (mode == kWaitFirst) asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (mode == kHintFirst) {
+    const int nh = min(st.n[inst], pol.budget - 1) + 1;
+    const int ch = ((nh + C - 1) / C + 1) & ~1;
+    const int lh = min(rank * ch, nh), cnth = min(lh + ch, nh) - lh;
+    const char* kb = reinterpret_cast<const char*>(st.K) + (inst * (size_t)pol.budget + lh) * (D * 2);
+    // only the head of the chunk: enough to cover the start-up latency without flooding L2
+    const int lines = min((cnth * D * 2) >> 7, kPrefetchLines);
+    for (int i = tid; i < lines; i += kThreads) {
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(kb + (size_t)i * 128));
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");         // counters, q, k_new, v_new are read after this
   }
   const int n0 = st.n[inst];
   const int tot = st.total[inst];
@@ -119,21 +138,37 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   const uint4* knew = reinterpret_cast<const uint4*>(k_new) + ((size_t)seq * kv_heads + head) * NCH;
   const uint4* vnew = reinterpret_cast<const uint4*>(v_new) + ((size_t)seq * kv_heads + head) * NCH;
 
-  if (early) {
-    const char* kb = reinterpret_cast<const char*>(Kc + (size_t)lo * NCH);
-    // only the head of the chunk: enough to cover the start-up latency without flooding L2
-    const int lines = min((cnt * NCH * 16) >> 7, kPrefetchLines);
-    for (int i = tid; i < lines; i += kThreads) {
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(kb + (size_t)i * 128));
-    }
-    asm volatile("griddepcontrol.wait;" ::: "memory");         // q, k_new, v_new and out belong to the caller's chain
-  }
-
   // The CTA whose chunk holds slot n0 stores the appended token (Eq. 2).
   if (n0 >= lo && n0 < hi) {
     if (tid < NCH) (reinterpret_cast<uint4*>(st.K) + cache_off)[(size_t)n0 * NCH + tid] = knew[tid];
     else if (tid < 2 * NCH) (reinterpret_cast<uint4*>(st.V) + cache_off)[(size_t)n0 * NCH + tid - NCH] = vnew[tid - NCH];
     else if (tid == 2 * NCH) st.pos[inst * pol.budget + n0] = tot;
+  }
+
+  // Rolling L2 prefetch. The CTA's traffic is one stream: its K rows, then its V rows, then (as a
+  // hint only) the head of the same chunk in the NEXT layer's K cache, which the next decode launch
+  // of a layer stack reads first; pulling that towards L2 while this kernel reduces and updates its
+  // scores keeps HBM busy across the launch boundary. Row index `vr` runs over that stream with each
+  // part padded to a multiple of the rows one loop iteration covers. One line per lane and tile.
+  constexpr int kIterRows = kWarps * kTile;
+  constexpr int kLinesPerRow = (D * 2) / 128;                  // 1 (d = 64) or 2 (d = 128)
+  const int cntR = (cnt + kIterRows - 1) / kIterRows * kIterRows;
+  const char* pfK = reinterpret_cast<const char*>(Kc + (size_t)lo * NCH);
+  const char* pfV = reinterpret_cast<const char*>(Vc + (size_t)lo * NCH);
+  const size_t inst_next = ((size_t)max(next_layer, 0) * max_batch + seq) * kv_heads + head;
+  const char* pfN = reinterpret_cast<const char*>(reinterpret_cast<const uint4*>(st.K) +
+                                                  (inst_next * (size_t)pol.budget + lo) * NCH);
+  auto prefetch_tile = [&](int vr) {
+    int row = vr + lane / kLinesPerRow;
+    if (lane >= kTile * kLinesPerRow) return;
+    const char* b = pfK;
+    if (vr >= 2 * cntR) { if (next_layer < 0) return; row -= 2 * cntR; b = pfN; }
+    else if (vr >= cntR) { row -= cntR; b = pfV; }
+    if (row < cnt) asm volatile("prefetch.global.L2 [%0];" ::"l"(b + (size_t)row * (D * 2) + (lane % kLinesPerRow) * 128));
+  };
+  {   // this chunk's score words are read at the very end: start them towards L2 now
+    const char* sb = reinterpret_cast<const char*>(st.score + inst * pol.budget + lo);
+    if (tid * 128 < cnt * 4) asm volatile("prefetch.global.L2 [%0];" ::"l"(sb + (size_t)tid * 128));
   }
 
   // ---- phase 1: logits, S^T = K Q^T ------------------------------------------------------
@@ -160,6 +195,7 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
     for (int base = warp * kTile; base < cnt; base += kWarps * kTile) {
       const int ra = base + r8, rb = base + r8 + 8;
       load_k(base + kWarps * kTile, ka2, kb2);    // next tile's loads are in flight during the MMAs
+      if (kAhead > 0) prefetch_tile(base + (kAhead + 1) * kIterRows);
       float s[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int i = 0; i < KL; ++i)
@@ -180,6 +216,18 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
       for (int i = 0; i < KL; ++i) { ka[i] = ka2[i]; kb[i] = kb2[i]; }
     }
   }
+  auto load_v = [&](int base, uint4 (&vv)[4][VJ]) {
+    const int row[4] = {base + 2 * c4, base + 2 * c4 + 1, base + 2 * c4 + 8, base + 2 * c4 + 9};
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const uint4* p = (lo + row[x] == n0) ? vnew : Vc + (size_t)(lo + row[x]) * NCH;
+#pragma unroll
+      for (int j = 0; j < VJ; ++j)
+        vv[x][j] = (row[x] < cnt) ? ld_stream(p + r8 + 8 * j) : make_uint4(0, 0, 0, 0);
+    }
+  };
+  uint4 vv[4][VJ], vn[4][VJ];
+  load_v(warp * kTile, vv);                      // in flight across the reduction of the maxima
 #pragma unroll
   for (int e = 0; e < 2; ++e) {
 #pragma unroll
@@ -206,21 +254,10 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
 #pragma unroll
         for (int e = 0; e < 4; ++e) oc[j][jj][e] = 0.f;
     const float mh = (r8 < G) ? mloc[r8] : 0.f;
-    auto load_v = [&](int base, uint4 (&vv)[4][VJ]) {
-      const int row[4] = {base + 2 * c4, base + 2 * c4 + 1, base + 2 * c4 + 8, base + 2 * c4 + 9};
-#pragma unroll
-      for (int x = 0; x < 4; ++x) {
-        const uint4* p = (lo + row[x] == n0) ? vnew : Vc + (size_t)(lo + row[x]) * NCH;
-#pragma unroll
-        for (int j = 0; j < VJ; ++j)
-          vv[x][j] = (row[x] < cnt) ? ld_stream(p + r8 + 8 * j) : make_uint4(0, 0, 0, 0);
-      }
-    };
-    uint4 vv[4][VJ], vn[4][VJ];
-    load_v(warp * kTile, vv);
     for (int base = warp * kTile; base < cnt; base += kWarps * kTile) {
       const int row[4] = {base + 2 * c4, base + 2 * c4 + 1, base + 2 * c4 + 8, base + 2 * c4 + 9};
       load_v(base + kWarps * kTile, vn);
+      if (kAhead > 0) prefetch_tile(cntR + base + (kAhead + 1) * kIterRows);
       // P^T fragment: head r8, keys base + 2*c4 + {0,1} and + 8
       float p0 = 0.f, p1 = 0.f, p2 = 0.f, p3 = 0.f;
       if (r8 < G) {
@@ -289,6 +326,7 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
 
   // ---- combine across the cluster -------------------------------------------------------
   cluster.sync();
+  if (mode == kOverlap) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (rank == 0 && tid == 0) {       // every CTA has read n0/tot before the barrier
     st.n[inst] = n1;
     st.total[inst] = tot + 1;
@@ -332,7 +370,7 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
 
 template <int D, int G>
 cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, const void* v_new,
-                   void* out, int cluster_size, int early, cudaStream_t stream) {
+                   void* out, int cluster_size, int mode, int next_layer, cudaStream_t stream) {
   const int batch = c->batch[layer];
   const int chunk_cap = (((c->pol.budget + cluster_size - 1) / cluster_size + 1) & ~1) + 2;
   const size_t smem = sizeof(Partial<G, D>) +
@@ -363,17 +401,17 @@ cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, con
   return cudaLaunchKernelEx(&cfg, decode_bf16_kernel<D, G>, c->st, c->pol, (const __nv_bfloat16*)q,
                             (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, (__nv_bfloat16*)out,
                             layer, c->sh.max_batch, c->sh.kv_heads, chunk_cap, scale_log2,
-                            (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0, early);
+                            (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0, mode, next_layer);
 }
 
 template <int D>
 cudaError_t launch_g(buzz_ctx* c, int layer, const void* q, const void* k_new, const void* v_new,
-                     void* out, int cs, int early, cudaStream_t stream) {
+                     void* out, int cs, int mode, int next_layer, cudaStream_t stream) {
   switch (c->group) {
-    case 1: return launch<D, 1>(c, layer, q, k_new, v_new, out, cs, early, stream);
-    case 2: return launch<D, 2>(c, layer, q, k_new, v_new, out, cs, early, stream);
-    case 4: return launch<D, 4>(c, layer, q, k_new, v_new, out, cs, early, stream);
-    case 8: return launch<D, 8>(c, layer, q, k_new, v_new, out, cs, early, stream);
+    case 1: return launch<D, 1>(c, layer, q, k_new, v_new, out, cs, mode, next_layer, stream);
+    case 2: return launch<D, 2>(c, layer, q, k_new, v_new, out, cs, mode, next_layer, stream);
+    case 4: return launch<D, 4>(c, layer, q, k_new, v_new, out, cs, mode, next_layer, stream);
+    case 8: return launch<D, 8>(c, layer, q, k_new, v_new, out, cs, mode, next_layer, stream);
     default: return cudaErrorInvalidValue;
   }
 }
@@ -381,7 +419,8 @@ cudaError_t launch_g(buzz_ctx* c, int layer, const void* q, const void* k_new, c
 }  // namespace
 
 cudaError_t buzz_launch_decode_bf16(buzz_ctx* c, int layer, const void* q, const void* k_new,
-                                    const void* v_new, void* out, int cluster_size, int early, cudaStream_t stream) {
-  return c->sh.head_dim == 128 ? launch_g<128>(c, layer, q, k_new, v_new, out, cluster_size, early, stream)
-                               : launch_g<64>(c, layer, q, k_new, v_new, out, cluster_size, early, stream);
+                                    const void* v_new, void* out, int cluster_size, int mode, int next_layer,
+                                    cudaStream_t stream) {
+  return c->sh.head_dim == 128 ? launch_g<128>(c, layer, q, k_new, v_new, out, cluster_size, mode, next_layer, stream)
+                               : launch_g<64>(c, layer, q, k_new, v_new, out, cluster_size, mode, next_layer, stream);
 }

@@ -91,7 +91,7 @@ def check_prefill_sampled(w, Q, K, V, got, gpu_scores, rows, tail_keys, tol, log
 
 def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None, check_every=1,
                  device="cuda:0", logn=False, bz: Buzz | None = None, sampled_rows=None, tail_keys=64,
-                 sampling=None):
+                 sampling=None, layers_call=False):
     """Runs prefill + decode/evict on the GPU for the whole workload and the oracle on `samples`
     (a list of (layer, seq, kv_head)). Returns a dict of summary counters."""
     tol = TOL[w.dtype]
@@ -147,12 +147,14 @@ def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None,
             compare_state(bz, ls, layer, b, h, f"after prefill L{layer} b{b} h{h}", exact_scores=True)
             lock[(layer, b, h)] = ls
     for t in range(S):
-        outs = {}
-        for layer in layers:
-            qd, kd, vd = dec[layer]
-            o = torch.empty_like(qd[t])
-            bz.decode_step(layer, qd[t], kd[t], vd[t], o)
-            outs[layer] = o
+        outs = {layer: torch.empty_like(dec[layer][0][t]) for layer in layers}
+        if layers_call:                          # the whole stack in one multi-layer call
+            bz.decode_layers(layers, [dec[l][0][t] for l in layers], [dec[l][1][t] for l in layers],
+                             [dec[l][2][t] for l in layers], [outs[l] for l in layers])
+        else:
+            for layer in layers:
+                qd, kd, vd = dec[layer]
+                bz.decode_step(layer, qd[t], kd[t], vd[t], outs[layer])
         pre = {}
         for key, ls in lock.items():
             layer, b, h = key

@@ -17,12 +17,14 @@ def test_c1_full(cuda_device):
     assert stats["prefill_rounds"] == 1 and stats["evictions"] == 3
 
 
-def test_c2_shape_scaled(cuda_device):
+@pytest.mark.parametrize("layers_call", [False, True])
+def test_c2_shape_scaled(cuda_device, layers_call):
     """Llama-2-7B head shape (bf16, d=128, MHA), low-rank + outlier keys; several key tiles and a
-    ragged tail; budget small enough that decode-time evictions happen."""
+    ragged tail; budget small enough that decode-time evictions happen. Run once with one decode
+    call per layer and once with the whole stack in one multi-layer call."""
     w = workloads.scaled(workloads.get("C2"), layers=2, batch=3, q_heads=4, kv_heads=4,
                          prompt_min=700, prompt_max=700, decode_steps=150, window=64, budget=180)
-    stats = run_lockstep(w, [(0, 0, 0), (0, 2, 3), (1, 1, 2)], check_every=7)
+    stats = run_lockstep(w, [(0, 0, 0), (0, 2, 3), (1, 1, 2)], check_every=7, layers_call=layers_call)
     assert stats["prefill_rounds"] >= 1 and stats["evictions"] >= 3
 
 
@@ -303,3 +305,103 @@ def test_decode_step_host_matches_device_entry(cuda_device):
         assert bz.status() == 0
     for bz in (ref, sep, packed):
         bz.close()
+
+
+def _stack(w, device="cuda:0"):
+    pre = [workloads.prefill_inputs(w, l, device) for l in range(w.layers)]
+    dec = [workloads.decode_inputs(w, l, device) for l in range(w.layers)]
+    return pre, dec
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("shape", [dict(batch=2, q_heads=8, kv_heads=2), dict(batch=1, q_heads=2, kv_heads=2),
+                                   dict(batch=3, q_heads=16, kv_heads=16)])
+def test_decode_layers_matches_single_layer_calls(cuda_device, shape):
+    """One multi-layer call per step (device pointers, and packed host buffers) leaves bit-identical
+    outputs, scores and caches to one buzz_decode_step per layer, across evictions, for any order of
+    the layers, with and without an eviction call between steps."""
+    w = workloads.scaled(workloads.get("C4"), layers=4, prompt_min=150, prompt_max=150, decode_steps=40,
+                         window=32, budget=180, **shape)
+    pre, dec = _stack(w)
+    ref, multi, host = make_buzz(w), make_buzz(w), make_buzz(w)
+    for bz in (ref, multi, host):
+        for l in range(w.layers):
+            q, k, v, cu = pre[l]
+            bz.prefill(l, q, k, v, cu, 150, torch.empty_like(q))
+    orders = [[0, 1, 2, 3], [3, 1, 0, 2], [2, 0, 3, 1]]
+    for t in range(w.decode_steps):
+        order = orders[t % 3]
+        o_ref = {l: torch.empty_like(dec[l][0][t]) for l in order}
+        for l in order:
+            ref.decode_step(l, dec[l][0][t], dec[l][1][t], dec[l][2][t], o_ref[l])
+        o_m = {l: torch.empty_like(dec[l][0][t]) for l in order}
+        multi.decode_layers(order, [dec[l][0][t] for l in order], [dec[l][1][t] for l in order],
+                            [dec[l][2][t] for l in order], [o_m[l] for l in order])
+        rec = torch.cat([torch.cat([dec[l][i][t].reshape(-1) for i in range(3)]) for l in order]).cpu().pin_memory()
+        o_h = torch.empty(sum(o_ref[l].numel() for l in order), dtype=rec.dtype).pin_memory()
+        host.decode_layers_host(order, rec, o_h)
+        if t % 2 == 0:                       # on odd steps the next call follows the last one directly
+            for bz in (ref, multi, host):
+                bz.evict(-1)
+        torch.cuda.synchronize()
+        flat = torch.cat([o_ref[l].reshape(-1) for l in order]).cpu()
+        assert torch.equal(torch.cat([o_m[l].reshape(-1) for l in order]).cpu(), flat), f"step {t}"
+        assert torch.equal(o_h, flat), f"host entry, step {t}"
+    for bz in (multi, host):
+        for l in range(w.layers):
+            for b in range(w.batch):
+                a, c = ref.export_state(l, b, w.kv_heads - 1), bz.export_state(l, b, w.kv_heads - 1)
+                assert (a["n"], a["n_old"], a["total_len"]) == (c["n"], c["n_old"], c["total_len"])
+                assert torch.equal(a["pos"], c["pos"]) and torch.equal(a["score"], c["score"])
+                assert torch.equal(a["k"], c["k"]) and torch.equal(a["v"], c["v"])
+        assert bz.status() == 0
+    for bz in (ref, multi, host):
+        bz.close()
+
+
+@pytest.mark.gpu
+def test_two_small_layers_alternating_without_eviction_calls(cuda_device):
+    """Small grids let several launches be resident at once. Alternating two layers call after call,
+    with nothing between the calls, must give what fully serialised calls give."""
+    w = workloads.scaled(workloads.get("C4"), layers=2, batch=1, q_heads=4, kv_heads=1, prompt_min=100,
+                         prompt_max=100, decode_steps=60, window=16, budget=400)
+    pre, dec = _stack(w)
+    ref, fast = make_buzz(w), make_buzz(w)
+    for bz in (ref, fast):
+        for l in range(2):
+            q, k, v, cu = pre[l]
+            bz.prefill(l, q, k, v, cu, 100, torch.empty_like(q))
+    o_ref = [[torch.empty_like(dec[l][0][t]) for l in range(2)] for t in range(w.decode_steps)]
+    o_fast = [[torch.empty_like(dec[l][0][t]) for l in range(2)] for t in range(w.decode_steps)]
+    for t in range(w.decode_steps):
+        for l in range(2):
+            ref.decode_step(l, dec[l][0][t], dec[l][1][t], dec[l][2][t], o_ref[t][l])
+            torch.cuda.synchronize()
+    for t in range(w.decode_steps):              # enqueued back to back, no synchronisation
+        for l in range(2):
+            fast.decode_step(l, dec[l][0][t], dec[l][1][t], dec[l][2][t], o_fast[t][l])
+    torch.cuda.synchronize()
+    for t in range(w.decode_steps):
+        for l in range(2):
+            assert torch.equal(o_ref[t][l], o_fast[t][l]), f"step {t} layer {l}"
+    for l in range(2):
+        a, c = ref.export_state(l, 0, 0), fast.export_state(l, 0, 0)
+        assert a["n"] == c["n"] == 160 and torch.equal(a["score"], c["score"])
+    ref.close(); fast.close()
+
+
+@pytest.mark.gpu
+def test_decode_layers_rejects_bad_layer_lists(cuda_device):
+    from paper_2410_23079_b200 import BuzzError
+    w = workloads.scaled(workloads.get("C4"), layers=2, batch=1, q_heads=4, kv_heads=1, prompt_min=64,
+                         prompt_max=64, decode_steps=1, window=16, budget=100)
+    bz = make_buzz(w)
+    qd, kd, vd = workloads.decode_inputs(w, 0, "cuda:0")
+    o = torch.empty_like(qd[0])
+    for bad in ([0, 0], [0, 2], [-1], [0, 1, 0]):
+        n = len(bad)
+        with pytest.raises(BuzzError):
+            bz.decode_layers(bad, [qd[0]] * n, [kd[0]] * n, [vd[0]] * n, [o] * n)
+    with pytest.raises(BuzzError):
+        bz.decode_layers_host([1, 1], qd[0].cpu(), o.cpu())
+    bz.close()
