@@ -1,8 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the BUZZ hot path on B200: decode tokens/s with attention + eviction.
 
-A "step" is one decode step of the whole attention stack: for every layer ``buzz_decode_step``
-(append, attention over the compacted cache, score update), then ``buzz_evict`` for all layers.
+A "step" is one decode step of the whole attention stack: ``buzz_decode_layers`` over all layers
+(per layer: append, attention over the compacted cache, score update; one kernel launch per layer,
+the launches of a call overlap on the GPU), then ``buzz_evict`` for all layers.
 The caches are first filled by ``buzz_prefill`` of the workload's prompts (timed as its own leg and
 reported under ``prefill``); after the timed steps the run continues until the first decode-time
 eviction and times that call (``evict``).
@@ -147,6 +148,27 @@ class ClockSampler:
         return out
 
 
+def _warm_library(w, dt, dev):
+    """One throw-away pass of every kernel on a tiny object of the same head shape, so that module
+    loading and one-time attribute set-up are not charged to the first timed call."""
+    from paper_2410_23079_b200 import Buzz
+    n = 512
+    small = Buzz(sink=w.sink, window=w.window, segment=w.segment, hitters=w.hitters, budget=w.budget, layers=2,
+                 max_batch=1, q_heads=w.q_heads, kv_heads=w.kv_heads, head_dim=w.head_dim, dtype=dt,
+                 max_prompt_tokens=n, device=dev)
+    cu = torch.tensor([0, n], dtype=torch.int32, device=dev)
+    q = torch.randn((n, w.q_heads, w.head_dim), device=dev).to(dt)
+    k = torch.randn((n, w.kv_heads, w.head_dim), device=dev).to(dt)
+    for layer in range(2):
+        small.prefill(layer, q, k, k, cu, n, torch.empty_like(q))
+    o = [torch.empty_like(q[:1]) for _ in range(2)]
+    small.decode_layers([0, 1], [q[:1]] * 2, [k[:1]] * 2, [k[:1]] * 2, o)
+    small.evict(-1)
+    torch.cuda.synchronize()
+    assert small.status() == 0
+    small.close()
+
+
 def run_ours(args):
     from paper_2410_23079_b200 import Buzz
     rank = int(os.environ.get("RANK", 0))
@@ -171,6 +193,7 @@ def run_ours(args):
               layers=w.layers, max_batch=w.batch, q_heads=w.q_heads, kv_heads=w.kv_heads,
               head_dim=w.head_dim, dtype=dt, max_prompt_tokens=total, device=dev)
     stream = torch.cuda.current_stream()
+    _warm_library(w, dt, dev)
 
     # ---- prefill leg (fills the caches; timed per layer around the library call only) --------
     pre_ms = 0.0
@@ -200,10 +223,11 @@ def run_ours(args):
     outs = [torch.empty_like(dec[layer][0][0]) for layer in range(w.layers)]
     counts = [_after_prefill(n, w) for n in lens]
 
+    all_layers = list(range(w.layers))
+
     def step(t):
-        for layer in range(w.layers):
-            qd, kd, vd = dec[layer]
-            bz.decode_step(layer, qd[t % pool], kd[t % pool], vd[t % pool], outs[layer])
+        i = t % pool
+        bz.decode_layers(all_layers, [d[0][i] for d in dec], [d[1][i] for d in dec], [d[2][i] for d in dec], outs)
 
     def advance_counts():
         nonlocal counts
@@ -265,22 +289,21 @@ def run_ours(args):
 
     # ---- end-to-end leg: the same step through the host-buffer entry point -------------------
     Ke = min(K, args.e2e_steps)
-    # pinned host inputs, one packed q|k|v record per (layer, step) so that a step's inputs go down in one copy
+    # pinned host inputs: per step one packed buffer, for each layer q | k_new | v_new, so that a step's
+    # inputs go down in one copy and its outputs come back in one
     nq = w.batch * w.q_heads * w.head_dim
     nk = w.batch * w.kv_heads * w.head_dim
-    hin = [torch.empty((pool, nq + 2 * nk), dtype=dt).pin_memory() for l in range(w.layers)]
-    ho = [torch.empty(tuple(dec[l][0].shape[1:]), dtype=dt).pin_memory() for l in range(w.layers)]
+    hin = torch.empty((pool, w.layers, nq + 2 * nk), dtype=dt).pin_memory()
+    ho = torch.empty((w.layers, nq), dtype=dt).pin_memory()
     for l in range(w.layers):
-        hin[l][:, :nq].copy_(dec[l][0].reshape(pool, nq))
-        hin[l][:, nq:nq + nk].copy_(dec[l][1].reshape(pool, nk))
-        hin[l][:, nq + nk:].copy_(dec[l][2].reshape(pool, nk))
+        hin[:, l, :nq].copy_(dec[l][0].reshape(pool, nq))
+        hin[:, l, nq:nq + nk].copy_(dec[l][1].reshape(pool, nk))
+        hin[:, l, nq + nk:].copy_(dec[l][2].reshape(pool, nk))
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for i in range(Ke):
-        for layer in range(w.layers):
-            rec = hin[layer][t % pool]
-            bz.decode_step_host(layer, rec[:nq], rec[nq:nq + nk], rec[nq + nk:], ho[layer])
+        bz.decode_layers_host(all_layers, hin[t % pool], ho)
         bz.evict(-1)
         advance_counts(); t += 1
     e1.record(stream)

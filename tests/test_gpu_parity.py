@@ -340,7 +340,7 @@ def test_decode_layers_matches_single_layer_calls(cuda_device, shape):
         rec = torch.cat([torch.cat([dec[l][i][t].reshape(-1) for i in range(3)]) for l in order]).cpu().pin_memory()
         o_h = torch.empty(sum(o_ref[l].numel() for l in order), dtype=rec.dtype).pin_memory()
         host.decode_layers_host(order, rec, o_h)
-        if t % 2 == 0:                       # on odd steps the next call follows the last one directly
+        if t % 2 == 0 or t >= 20:            # early odd steps: the next call follows the last one directly
             for bz in (ref, multi, host):
                 bz.evict(-1)
         torch.cuda.synchronize()
