@@ -33,11 +33,8 @@ constexpr int kMaxCluster = 8;
 constexpr int kHeads = 8;       // MMA column count: query heads of one group, zero-padded
 constexpr int kTile = 16;       // keys per warp tile
 constexpr int kPrefetchLines = 256;   // 128-byte lines of K a CTA may pull towards L2 before its wait (measured best)
-#ifndef BUZZ_DECODE_PD
-#define BUZZ_DECODE_PD 2
-#endif
 enum { kWaitFirst = 0, kHintFirst = 1, kOverlap = 2 };
-constexpr int kAhead = BUZZ_DECODE_PD;   // rolling L2 prefetch distance, in loop iterations (kWarps * kTile rows each)
+constexpr int kAhead = 2;   // rolling L2 prefetch runs this many loop iterations (kWarps * kTile rows each) ahead of the register loads (measured best of 0..5)
 
 __device__ inline uint4 ld_stream(const uint4* p) { return __ldcs(p); }
 
