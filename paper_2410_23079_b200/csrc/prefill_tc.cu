@@ -235,7 +235,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 // logits that reuse an S buffer are only issued once both P V products on it have been seen to
 // complete (pv_done).
 // =================================================================================================
-constexpr int kThreadsA = 320;            // TMA warp, MMA warp, 2 x 4 softmax warps
+constexpr int kThreadsA = 352;            // TMA warp, Q K^T issuer, 2 x 4 softmax warps, P V issuer
 constexpr int kStagesA = 3;
 struct SmemA {
   alignas(1024) unsigned char q[kTileBytes];
@@ -307,12 +307,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
   } else if (warp == 1) {
-    // ---- MMA issuer ----
+    // ---- Q K^T issuer: S[j%2] = Q K_j^T, one tile ahead of the softmax ----
+    // The two products are issued by two different warps: the serial work of one issuing thread
+    // (five barrier waits and sixteen instruction issues per tile) was the longest chain in the loop.
     if (elect_one()) {
       const uint32_t qa = smem_u32(sm.q);
-      auto issue_qk = [&](int j) -> bool {             // S[j%2] = Q K_j^T
+      bool ok = mbar_wait(&sm.q_full, 0);
+      if (!ok) tf.raise(14);
+      for (int j = 0; ok && j < nt; ++j) {
         const int st = j % kStagesA;
-        if (!mbar_wait(&sm.k_full[st], (j / kStagesA) & 1)) { tf.raise(13); return false; }
+        if (!mbar_wait(&sm.k_full[st], (j / kStagesA) & 1)) { tf.raise(13); break; }
+        // S[j%2] still holds P of tile j-2: both of its P V products must have completed
+        if (j >= 2 && !mbar_wait(&sm.pv_done[j & 1], ((j - 2) >> 1) & 1)) { tf.raise(21); break; }
         tc_fence_after();
         const uint32_t ka = smem_u32(sm.k[st]);
 #pragma unroll
@@ -320,24 +326,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           mma_ss(tmem + (j & 1) * BT, kmajor_desc(qa, s), kmajor_desc(ka, s), kIdescKK, s > 0);
         mma_commit(&sm.s_full[j & 1]);
         mma_commit(&sm.k_empty[st]);
-        return true;
-      };
-      bool ok = mbar_wait(&sm.q_full, 0);
-      if (!ok) tf.raise(14);
-      ok = ok && issue_qk(0);
-      for (int j = 0; ok && j < nt; ++j) {
-        if (j + 1 < nt) {
-          // S[(j+1)%2] still holds P of tile j-1: both of its P V products must have completed
-          if (j >= 1 && !mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(21); break; }
-          if (!issue_qk(j + 1)) break;                 // next tile's logits overlap this tile's softmax
-        }
+      }
+    }
+  } else if (warp == 10) {
+    // ---- P V issuer: O_g += P_g V[64g .. 64g+63], 16 keys per step ----
+    if (elect_one()) {
+      for (int j = 0; j < nt; ++j) {
         const int sb = j & 1, st = j % kStagesA;
+        if (!mbar_wait(&sm.v_full[st], (j / kStagesA) & 1)) { tf.raise(16); break; }
+        const uint32_t va = smem_u32(sm.v[st]);
         bool fine = true;
-        for (int g = 0; g < 2 && fine; ++g) {          // O_g += P_g V[64g .. 64g+63], 16 keys per step
+        for (int g = 0; g < 2 && fine; ++g) {
           if (!mbar_wait(&sm.p_full[sb][g], (j >> 1) & 1)) { tf.raise(15); fine = false; break; }
-          if (g == 0 && !mbar_wait(&sm.v_full[st], (j / kStagesA) & 1)) { tf.raise(16); fine = false; break; }
           tc_fence_after();
-          const uint32_t va = smem_u32(sm.v[st]);
 #pragma unroll
           for (int s = 0; s < 4; ++s)
             mma_ts(tmem + kColO + g * BT, tmem + sb * BT + g * 64 + s * 8, mnmajor_desc(va, g * 4 + s), kIdescKM,
