@@ -35,6 +35,12 @@ constexpr float kInvLn512 = 1.0f / 6.2383246250395077f;
 constexpr uint32_t kIdescKK = idesc_bf16(BT, BT, false, false);   // both operands K-major
 constexpr uint32_t kIdescKM = idesc_bf16(BT, BT, false, true);    // B operand MN-major (V)
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 struct TimeoutFlag {
   int32_t* status;
   int inst;
@@ -248,7 +254,6 @@ struct SmemA {
 constexpr uint32_t kColO = 256;
 constexpr float kRescaleThreshold = 20.0f;    // log2: rescale O only when a row max grows by > 2^20
                                               // (P, the row sums and O stay far inside the fp32/bf16 exponent range)
-constexpr float kSpeculationLimit = 1048576.0f;   // 2^kRescaleThreshold: largest probability a speculative pass may produce
 
 __global__ void __launch_bounds__(kThreadsA, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -366,81 +371,60 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const uint32_t colS = sb * BT + g * 64;
       if (!mbar_wait(&sm.s_full[sb], (j >> 1) & 1)) { tf.raise(17); ok = false; break; }
       tc_fence_after();
-      // The raw logits of this half row. P is first formed SPECULATIVELY with the maximum in use (the
-      // output is only rescaled when a row maximum grows by more than 2^kRescaleThreshold, which after
-      // the first tiles is rare), and the largest probability is tracked alongside the exponentials,
-      // whose unit is the bottleneck, instead of in a pass of its own before them. Only if some row of
-      // the warp saw a probability above the threshold (or on the first tile, which has no maximum
-      // yet) are the logits read again from TMEM, the maximum taken properly and P formed again.
+      // the raw logits of this half row (rs > 0, so the maximum can be taken before scaling)
       float s[64];
-      auto load_logits = [&]() {
-        tmem_ld32(tmem + lane_base + colS, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-        tmem_ld32(tmem + lane_base + colS + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
-        tmem_wait_ld();
-        if (j == nt - 1) {                             // the diagonal tile: causal mask
+      tmem_ld32(tmem + lane_base + colS, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+      tmem_ld32(tmem + lane_base + colS + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+      tmem_wait_ld();
+      if (j == nt - 1) {                               // the diagonal tile: causal mask
 #pragma unroll
-          for (int c = 0; c < 64; ++c)
-            if (j * BT + g * 64 + c > qpos) s[c] = -INFINITY;
-        }
-      };
-      uint32_t pk[32];
-      float lsum = 0.f, pmax = 0.f;
-      auto exp_pass = [&]() {                          // P_g = 2^(S rs - m) as bf16 pairs, their sum and maximum
-        const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-        float l4[4] = {0.f, 0.f, 0.f, 0.f};
-        float x4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          const float p0 = exp2f(fmaf(s[2 * c], rs, neg_m));
-          const float p1 = exp2f(fmaf(s[2 * c + 1], rs, neg_m));
-          l4[c & 3] += p0 + p1;
-          x4[c & 3] = fmaxf(x4[c & 3], fmaxf(p0, p1));
-          const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
-          pk[c] = *reinterpret_cast<const uint32_t*>(&pp);
-        }
-        lsum = (l4[0] + l4[1]) + (l4[2] + l4[3]);
-        pmax = fmaxf(fmaxf(x4[0], x4[1]), fmaxf(x4[2], x4[3]));
-      };
-      load_logits();
-      bool settled = false;
-      if (j > 0) {
-        exp_pass();
-        // !(pmax <= limit) also catches an overflow to infinity
-        settled = !__any_sync(0xffffffffu, !(pmax <= kSpeculationLimit));
+        for (int c = 0; c < 64; ++c)
+          if (j * BT + g * 64 + c > qpos) s[c] = -INFINITY;
       }
-      if (!settled) {
-        if (j > 0) load_logits();                      // the speculative pass consumed the registers
-        float mx4[4] = {s[0], s[1], s[2], s[3]};       // rs > 0, so the maximum can be taken before scaling
+      float mx4[4] = {s[0], s[1], s[2], s[3]};         // four chains of three-input maxima
 #pragma unroll
-        for (int c = 4; c < 64; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], s[c]);
-        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * rs;   // -inf if the half row is masked out
-        const float m_new = fmaxf(m_used, mx);
-        if (j == 0) {
-          m_used = m_new;
-        } else {
-          const bool need = m_new > m_used + kRescaleThreshold;
-          if (__any_sync(0xffffffffu, need)) {
-            const float alpha = need ? exp2f(m_used - m_new) : 1.0f;     // 0 when nothing was unmasked so far
-            if (need) m_used = m_new;
-            l *= alpha;
-            if (!mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
-            tc_fence_after();
+      for (int c = 4; c < 64; c += 8) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) mx4[e] = max3(mx4[e], s[c + 2 * e], s[c + 2 * e + 1]);
+      }
+      const float mx = fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]) * rs;   // -inf if the half row is masked out
+      const float m_new = fmaxf(m_used, mx);
+      if (j == 0) {
+        m_used = m_new;
+      } else {
+        const bool need = m_new > m_used + kRescaleThreshold;
+        if (__any_sync(0xffffffffu, need)) {
+          const float alpha = need ? exp2f(m_used - m_new) : 1.0f;     // 0 when nothing was unmasked so far
+          if (need) m_used = m_new;
+          l *= alpha;
+          if (!mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
+          tc_fence_after();
 #pragma unroll 1
-            for (int c0 = 0; c0 < D; c0 += 32) {
-              uint32_t r[32];
-              tmem_ld32(tmem + lane_base + colOg + c0, r);
-              tmem_wait_ld();
+          for (int c0 = 0; c0 < D; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(tmem + lane_base + colOg + c0, r);
+            tmem_wait_ld();
 #pragma unroll
-              for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
-              tmem_st32(tmem + lane_base + colOg + c0, r);
-            }
-            tmem_wait_st();
+            for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
+            tmem_st32(tmem + lane_base + colOg + c0, r);
           }
+          tmem_wait_st();
         }
-        exp_pass();
       }
-      l += lsum;
+      // P_g = 2^(S rs - m) as bf16 pairs over the first 32 columns of this half row (which is in registers)
+      const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+      float l4[4] = {0.f, 0.f, 0.f, 0.f};
+      uint32_t pk[32];
+#pragma unroll
+      for (int c = 0; c < 32; ++c) {
+        const float p0 = exp2f(fmaf(s[2 * c], rs, neg_m));
+        const float p1 = exp2f(fmaf(s[2 * c + 1], rs, neg_m));
+        l4[c & 3] += p0 + p1;
+        const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
+        pk[c] = *reinterpret_cast<const uint32_t*>(&pp);
+      }
       tmem_st32(tmem + lane_base + colS, pk);
+      l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&sm.p_full[sb][g]);
