@@ -143,12 +143,13 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       prefetch_tensormap(&map_k);
       mbar_expect_tx(&sm.k_full, kTileBytes);
       load_tile(sm.k, &map_k, kvh * D, tok0 + key0, &sm.k_full);
+      int pg = 0, pqt = kt;
       for (int it = 0; it < iters; ++it) {
         const int st = it & 1, use = it >> 1;
         if (use > 0 && !mbar_wait(&sm.q_empty[st], (use - 1) & 1)) { tf.raise(1); break; }
-        const int g = it / nq, qt = kt + it % nq;
         mbar_expect_tx(&sm.q_full[st], kTileBytes);
-        load_tile(sm.q[st], &map_q, (kvh * G + g) * D, tok0 + qt * BT, &sm.q_full[st]);
+        load_tile(sm.q[st], &map_q, (kvh * G + pg) * D, tok0 + pqt * BT, &sm.q_full[st]);
+        if (++pqt == q_tiles) { pqt = kt; ++pg; }
       }
     }
   } else if (warp == 1) {
@@ -180,15 +181,17 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     // row statistics of tile `it` for this warp's 64 columns (two per lane): fetched from global
     // memory one iteration ahead, so the load's latency hides behind the previous tile's exponentials
     const int cw = warp - 2;                          // compute warp 0..7
-    auto fetch_lse = [&](int it, int e) -> float {
-      if (it >= iters) return 0.f;
-      const int qpos = (kt + it % nq) * BT + g * 64 + lane + 32 * e;
-      return (qpos < N) ? lse[(size_t)(kvh * G + it / nq) * stride + tok0 + qpos] : 0.f;
+    // (head of the group, query tile) of an iteration advance together; no divisions in the loop
+    auto fetch_lse = [&](int head, int tile, int e) -> float {
+      const int qpos = tile * BT + g * 64 + lane + 32 * e;
+      return (head < G && qpos < N) ? lse[(size_t)(kvh * G + head) * stride + tok0 + qpos] : 0.f;
     };
-    float lse_next0 = fetch_lse(0, 0), lse_next1 = fetch_lse(0, 1);
+    int qt = kt, nhead = 0, ntile = kt;                // this iteration's tile; next iteration's (head, tile)
+    float lse_next0 = fetch_lse(0, kt, 0), lse_next1 = fetch_lse(0, kt, 1);
     for (int it = 0; it < iters; ++it) {
       const int st = it & 1, use = it >> 1;
-      const int qt = kt + it % nq;
+      qt = ntile;
+      if (++ntile == q_tiles) { ntile = kt; ++nhead; }
       const int q0 = qt * BT;
       // this warp's private copy of the tile's row statistics (last read two iterations ago by this warp only)
       sm.lse[st][cw][lane] = lse_next0;
@@ -197,8 +200,8 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         sm.rs[st][cw][lane] = scale_log2 * __logf((float)(q0 + g * 64 + lane + 1)) * kInvLn512;
         sm.rs[st][cw][lane + 32] = scale_log2 * __logf((float)(q0 + g * 64 + lane + 33)) * kInvLn512;
       }
-      lse_next0 = fetch_lse(it + 1, 0);
-      lse_next1 = fetch_lse(it + 1, 1);
+      lse_next0 = fetch_lse(nhead, ntile, 0);
+      lse_next1 = fetch_lse(nhead, ntile, 1);
       __syncwarp();
       if (!mbar_wait(&sm.s_full[st], use & 1)) { tf.raise(5); ok = false; break; }
       tc_fence_after();
