@@ -66,7 +66,7 @@ __device__ __forceinline__ void load_tile(void* dst, const CUtensorMap* map, int
 // accumulators (column c -> acc[c % 4]), so the summation order is fixed and the adds pipeline.
 template <bool LOGN, int NC>
 __device__ __forceinline__ void colsum_tile(const uint32_t (&r)[NC], const float* __restrict__ rs,
-                                            const float* __restrict__ lse, float scale_log2, bool diag,
+                                            const float (&lse)[NC], float scale_log2, bool diag,
                                             bool tail, int q0, int kpos, int N, float (&acc)[4]) {
   if (!diag && !tail) {
 #pragma unroll
@@ -206,15 +206,27 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       if (!mbar_wait(&sm.s_full[st], use & 1)) { tf.raise(5); ok = false; break; }
       tc_fence_after();
       const bool diag = (qt == kt), tail = (q0 + BT > N);
-      // this thread's 64 logits first (two loads in flight), then 64 independent exponentials
-      uint32_t r[64];
-      tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + st * BT + g * 64, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
-      tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + st * BT + g * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
-      tmem_wait_ld();
-      tc_fence_before();
-      mbar_arrive(&sm.s_empty[st]);                    // S^T[st] may be overwritten once all 256 have arrived
-      if (logn) colsum_tile<true, 64>(r, sm.rs[st][cw], sm.lse[st][cw], scale_log2, diag, tail, q0 + g * 64, kpos, N, acc);
-      else colsum_tile<false, 64>(r, sm.rs[st][cw], sm.lse[st][cw], scale_log2, diag, tail, q0 + g * 64, kpos, N, acc);
+      // this thread's 64 logits in two halves of 32: the logits from TMEM and the columns' row statistics
+      // from shared memory (16-byte loads: memory instructions queue behind the exponentials), then 32
+      // independent exponentials
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        uint32_t r[32];
+        float ls[32];
+        tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + st * BT + g * 64 + h * 32, r);
+#pragma unroll
+        for (int c = 0; c < 32; c += 4) {
+          const float4 t = *reinterpret_cast<const float4*>(&sm.lse[st][cw][h * 32 + c]);
+          ls[c] = t.x; ls[c + 1] = t.y; ls[c + 2] = t.z; ls[c + 3] = t.w;
+        }
+        tmem_wait_ld();
+        if (h == 1) {
+          tc_fence_before();
+          mbar_arrive(&sm.s_empty[st]);                // S^T[st] may be overwritten once all 256 have arrived
+        }
+        if (logn) colsum_tile<true, 32>(r, sm.rs[st][cw] + h * 32, ls, scale_log2, diag, tail, q0 + g * 64 + h * 32, kpos, N, acc);
+        else colsum_tile<false, 32>(r, sm.rs[st][cw] + h * 32, ls, scale_log2, diag, tail, q0 + g * 64 + h * 32, kpos, N, acc);
+      }
       __syncwarp();                                   // the copy is rewritten two iterations from now
     }
     const float mine = (acc[0] + acc[1]) + (acc[2] + acc[3]);
