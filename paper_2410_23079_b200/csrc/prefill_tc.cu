@@ -243,52 +243,66 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 }
 
 // =================================================================================================
-// Pass A: attention output and row log-sum-exp. grid (query tiles, query heads, sequences), 1 CTA/SM.
-// The exponentials are the binding resource (16 per clock per SM; one warp per scheduler reaches a
-// quarter of that), so a query row is shared by TWO threads, one per softmax warpgroup: warpgroup g
-// owns key columns [64g, 64g+64) of every logits tile and runs a complete online softmax of its
-// own over them, with its own output accumulator (the P V product is split along the keys). The
-// warpgroups never synchronise inside the loop, so one can be taking maxima or waiting while the
-// other keeps the exponential unit busy; their (max, sum, output) are merged in the epilogue.
-//   TMEM columns: S0 [0,128)  S1 [128,256)  O_0 [256,384)  O_1 [384,512).
-// P_g (bf16 pairs, 32 columns) overwrites the start of the half row of S it was computed from.
-// The tensor core may still be reading P as the A operand long after the MMA was issued, so the
-// logits that reuse an S buffer are only issued once both P V products on it have been seen to
-// complete (pv_done).
+// Pass A: attention output and row log-sum-exp. grid (query tiles, query heads, sequences), TWO
+// CTAs per SM. A CTA owns 128 query rows and walks the keys in tiles of 64, one thread per row:
+//   TMEM columns (256 per CTA): S0 [0,64)  S1 [64,128)  O [128,256).
+// P (bf16 pairs, 32 columns) overwrites the start of the S buffer it was computed from. The
+// tensor core may still be reading P as the A operand long after the MMA was issued, so the
+// logits that reuse an S buffer are only issued once the P V product on it has been seen to
+// complete (pv_done). Inside one CTA the chain logits -> softmax -> P V -> next-but-one logits is
+// latency-bound (every barrier hand-over costs a few hundred cycles, more when the memory
+// instruction queue is full of exponentials); the second CTA on the SM fills those gaps, and
+// CTAs starting and finishing overlap with one in full flight.
+// Three warps do the asynchronous work: TMA producer, Q K^T issuer, P V issuer (one issuing
+// thread for both products was the longest serial chain in the loop).
 // =================================================================================================
-constexpr int kThreadsA = 352;            // TMA warp, Q K^T issuer, 2 x 4 softmax warps, P V issuer
-constexpr int kStagesA = 3;
+constexpr int KT = 64;                    // keys per tile in pass A
+constexpr uint32_t kKvBlockBytes = KT * 128;        // one [64 keys x 64 bf16] swizzled block
+constexpr uint32_t kKvTileBytes = 2 * kKvBlockBytes;
+constexpr int kThreadsA = 224;            // TMA warp, Q K^T issuer, 4 softmax warps, P V issuer
+constexpr int kStagesA = 2;
+constexpr uint32_t kIdescQK = idesc_bf16(BT, KT, false, false);
 struct SmemA {
   alignas(1024) unsigned char q[kTileBytes];
-  alignas(1024) unsigned char k[kStagesA][kTileBytes];
-  alignas(1024) unsigned char v[kStagesA][kTileBytes];
+  alignas(1024) unsigned char k[kStagesA][kKvTileBytes];
+  alignas(1024) unsigned char v[kStagesA][kKvTileBytes];
+  float xch[BT];
   uint64_t q_full, k_full[kStagesA], k_empty[kStagesA], v_full[kStagesA], v_empty[kStagesA];
-  uint64_t s_full[2], p_full[2][2], pv_done[2];
+  uint64_t s_full[2], p_full[2], pv_done[2];
   uint32_t tmem_base;
 };
-constexpr uint32_t kColO = 256;
+constexpr uint32_t kColO = 128;
 constexpr float kRescaleThreshold = 20.0f;    // log2: rescale O only when a row max grows by > 2^20
                                               // (P, the row sums and O stay far inside the fp32/bf16 exponent range)
 
-__global__ void __launch_bounds__(kThreadsA, 1)
+// K-major [64 keys][128 dims] tile as two swizzled blocks: descriptor of k-step ks (16 dims).
+__device__ __forceinline__ uint64_t kmajor_desc_kv(uint32_t tile_saddr, int ks) {
+  return smem_desc_sw128(tile_saddr + (ks >> 2) * kKvBlockBytes + (ks & 3) * 32, 16, 1024);
+}
+// MN-major V tile [64 keys][128 dims]: descriptor of k-step ks (16 keys), N = 128 dims.
+__device__ __forceinline__ uint64_t mnmajor_desc_kv(uint32_t tile_saddr, int ks) {
+  return smem_desc_sw128(tile_saddr + ks * 16 * 128, kKvBlockBytes, 1024);
+}
+__device__ __forceinline__ void load_kv_tile(void* dst, const CUtensorMap* map, int col0, int row0, uint64_t* bar) {
+  tma_load_2d(dst, map, col0, row0, bar);
+  tma_load_2d(static_cast<char*>(dst) + kKvBlockBytes, map, col0 + 64, row0, bar);
+}
+
+__global__ void __launch_bounds__(kThreadsA, 2)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const int32_t* __restrict__ cu,
                __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int32_t* status, int Hq, int Hkv,
                int stride, float scale_log2, int logn) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  SmemA& sm = *reinterpret_cast<SmemA*>(smem_raw);
+  SmemA& sm = *reinterpret_cast<SmemA*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int b = blockIdx.z, h = blockIdx.y, kvh = h / (Hq / Hkv);
   const int tok0 = cu[b], N = cu[b + 1] - tok0;
   const int qt = gridDim.x - 1 - blockIdx.x;          // heaviest (last) query tiles first
   const int row0 = qt * BT;
   if (row0 >= N) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nt = qt + 1;                              // key tiles 0..qt (causal)
+  const int nt = min(2 * qt + 2, (N + KT - 1) / KT);  // key tiles 0 .. (causal, clipped to the sequence)
   const TimeoutFlag tf{status, (b * Hq + h) * 4096 + qt};
-  if (smem_u32(smem_raw) & 1023u) {                   // the swizzled tiles need 1024-byte alignment
-    if (threadIdx.x == 0) buzz_set_status(status, BUZZ_ERR_INVALID, tf.inst, 30);
-    return;
-  }
 
   if (threadIdx.x == 0) {
     mbar_init(&sm.q_full, 1);
@@ -297,13 +311,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
     }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&sm.s_full[s], 1); mbar_init(&sm.pv_done[s], 1);
-      mbar_init(&sm.p_full[s][0], 128); mbar_init(&sm.p_full[s][1], 128);
+      mbar_init(&sm.s_full[s], 1); mbar_init(&sm.pv_done[s], 1); mbar_init(&sm.p_full[s], 128);
     }
     fence_barrier_init();
   }
   if (warp == 1) {
-    tmem_alloc(&sm.tmem_base, 512);
+    tmem_alloc(&sm.tmem_base, 256);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -320,17 +333,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       for (int j = 0; j < nt; ++j) {
         const int st = j % kStagesA, use = j / kStagesA;
         if (use > 0 && !mbar_wait(&sm.k_empty[st], (use - 1) & 1)) { tf.raise(11); break; }
-        mbar_expect_tx(&sm.k_full[st], kTileBytes);
-        load_tile(sm.k[st], &map_k, kvh * D, tok0 + j * BT, &sm.k_full[st]);
+        mbar_expect_tx(&sm.k_full[st], kKvTileBytes);
+        load_kv_tile(sm.k[st], &map_k, kvh * D, tok0 + j * KT, &sm.k_full[st]);
         if (use > 0 && !mbar_wait(&sm.v_empty[st], (use - 1) & 1)) { tf.raise(12); break; }
-        mbar_expect_tx(&sm.v_full[st], kTileBytes);
-        load_tile(sm.v[st], &map_v, kvh * D, tok0 + j * BT, &sm.v_full[st]);
+        mbar_expect_tx(&sm.v_full[st], kKvTileBytes);
+        load_kv_tile(sm.v[st], &map_v, kvh * D, tok0 + j * KT, &sm.v_full[st]);
       }
     }
   } else if (warp == 1) {
-    // ---- Q K^T issuer: S[j%2] = Q K_j^T, one tile ahead of the softmax ----
-    // The two products are issued by two different warps: the serial work of one issuing thread
-    // (five barrier waits and sixteen instruction issues per tile) was the longest chain in the loop.
+    // ---- Q K^T issuer: S[j%2] = Q K_j^T, up to two tiles ahead of the softmax ----
     if (elect_one()) {
       const uint32_t qa = smem_u32(sm.q);
       bool ok = mbar_wait(&sm.q_full, 0);
@@ -338,63 +349,56 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       for (int j = 0; ok && j < nt; ++j) {
         const int st = j % kStagesA;
         if (!mbar_wait(&sm.k_full[st], (j / kStagesA) & 1)) { tf.raise(13); break; }
-        // S[j%2] still holds P of tile j-2: both of its P V products must have completed
+        // S[j%2] still holds P of tile j-2: its P V product must have completed
         if (j >= 2 && !mbar_wait(&sm.pv_done[j & 1], ((j - 2) >> 1) & 1)) { tf.raise(21); break; }
         tc_fence_after();
         const uint32_t ka = smem_u32(sm.k[st]);
 #pragma unroll
         for (int s = 0; s < D / 16; ++s)
-          mma_ss(tmem + (j & 1) * BT, kmajor_desc(qa, s), kmajor_desc(ka, s), kIdescKK, s > 0);
+          mma_ss(tmem + (j & 1) * KT, kmajor_desc(qa, s), kmajor_desc_kv(ka, s), kIdescQK, s > 0);
         mma_commit(&sm.s_full[j & 1]);
         mma_commit(&sm.k_empty[st]);
       }
     }
-  } else if (warp == 10) {
-    // ---- P V issuer: O_g += P_g V[64g .. 64g+63], 16 keys per step ----
+  } else if (warp == 6) {
+    // ---- P V issuer: O += P V_j, 16 keys per step ----
     if (elect_one()) {
       for (int j = 0; j < nt; ++j) {
         const int sb = j & 1, st = j % kStagesA;
         if (!mbar_wait(&sm.v_full[st], (j / kStagesA) & 1)) { tf.raise(16); break; }
+        if (!mbar_wait(&sm.p_full[sb], (j >> 1) & 1)) { tf.raise(15); break; }
+        tc_fence_after();
         const uint32_t va = smem_u32(sm.v[st]);
-        bool fine = true;
-        for (int g = 0; g < 2 && fine; ++g) {
-          if (!mbar_wait(&sm.p_full[sb][g], (j >> 1) & 1)) { tf.raise(15); fine = false; break; }
-          tc_fence_after();
 #pragma unroll
-          for (int s = 0; s < 4; ++s)
-            mma_ts(tmem + kColO + g * BT, tmem + sb * BT + g * 64 + s * 8, mnmajor_desc(va, g * 4 + s), kIdescKM,
-                   (j > 0 || s > 0) ? 1u : 0u);
-        }
-        if (!fine) break;
+        for (int s = 0; s < KT / 16; ++s)
+          mma_ts(tmem + kColO, tmem + sb * KT + s * 8, mnmajor_desc_kv(va, s), kIdescKM, (j > 0 || s > 0) ? 1u : 0u);
         mma_commit(&sm.v_empty[st]);
         mma_commit(&sm.pv_done[sb]);
       }
     }
   } else {
-    // ---- softmax: thread (g, row) runs an online softmax over key columns [64g, 64g+64) of every tile ----
-    const int g = (warp - 2) >> 2;
+    // ---- softmax: one thread per query row, 64 logits per tile ----
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const int qpos = row0 + row;
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    const uint32_t colOg = kColO + g * BT;
     const float rs = scale_log2 * (logn ? __logf((float)(qpos + 1)) * kInvLn512 : 1.0f);
     float m_used = -INFINITY, l = 0.f;
     bool ok = true;
     for (int j = 0; j < nt; ++j) {
       const int sb = j & 1;
-      const uint32_t colS = sb * BT + g * 64;
+      const uint32_t colS = sb * KT;
       if (!mbar_wait(&sm.s_full[sb], (j >> 1) & 1)) { tf.raise(17); ok = false; break; }
       tc_fence_after();
-      // the raw logits of this half row (rs > 0, so the maximum can be taken before scaling)
+      // the raw logits of this row (rs > 0, so the maximum can be taken before scaling)
       float s[64];
       tmem_ld32(tmem + lane_base + colS, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
       tmem_ld32(tmem + lane_base + colS + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
       tmem_wait_ld();
-      if (j == nt - 1) {                               // the diagonal tile: causal mask
+      if (j * KT + KT - 1 > row0) {                    // a tile that crosses the diagonal: causal mask
 #pragma unroll
         for (int c = 0; c < 64; ++c)
-          if (j * BT + g * 64 + c > qpos) s[c] = -INFINITY;
+          if (j * KT + c > qpos) s[c] = -INFINITY;
       }
       float mx4[4] = {s[0], s[1], s[2], s[3]};         // four chains of three-input maxima
 #pragma unroll
@@ -402,14 +406,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll
         for (int e = 0; e < 4; ++e) mx4[e] = max3(mx4[e], s[c + 2 * e], s[c + 2 * e + 1]);
       }
-      const float mx = fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]) * rs;   // -inf if the half row is masked out
+      const float mx = fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]) * rs;   // -inf if the whole tile is masked for this row
       const float m_new = fmaxf(m_used, mx);
       if (j == 0) {
-        m_used = m_new;
+        m_used = m_new;                                // finite: key 0 is never masked
       } else {
         const bool need = m_new > m_used + kRescaleThreshold;
         if (__any_sync(0xffffffffu, need)) {
-          const float alpha = need ? exp2f(m_used - m_new) : 1.0f;     // 0 when nothing was unmasked so far
+          const float alpha = need ? exp2f(m_used - m_new) : 1.0f;
           if (need) m_used = m_new;
           l *= alpha;
           if (!mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
@@ -417,17 +421,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
 #pragma unroll 1
           for (int c0 = 0; c0 < D; c0 += 32) {
             uint32_t r[32];
-            tmem_ld32(tmem + lane_base + colOg + c0, r);
+            tmem_ld32(tmem + lane_base + kColO + c0, r);
             tmem_wait_ld();
 #pragma unroll
             for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
-            tmem_st32(tmem + lane_base + colOg + c0, r);
+            tmem_st32(tmem + lane_base + kColO + c0, r);
           }
           tmem_wait_st();
         }
       }
-      // P_g = 2^(S rs - m) as bf16 pairs over the first 32 columns of this half row (which is in registers)
-      const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+      // P = 2^(S rs - m) as bf16 pairs over the first 32 columns of this S buffer (S is in registers)
+      const float neg_m = -m_used;
       float l4[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pk[32];
 #pragma unroll
@@ -442,37 +446,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&sm.p_full[sb][g]);
+      mbar_arrive(&sm.p_full[sb]);
     }
-    // ---- epilogue: merge the two halves of the row, O / l -> bf16, row log2-sum-exp ----
+    // ---- epilogue: O / l -> bf16, row log2-sum-exp ----
     if (ok && !mbar_wait(&sm.pv_done[(nt - 1) & 1], ((nt - 1) >> 1) & 1)) { tf.raise(19); ok = false; }
     tc_fence_after();
-    // the K ring is idle now (its last use completed before that P V product): exchange (max, sum) there
-    float* xm = reinterpret_cast<float*>(sm.k[0]);    // [2][BT]
-    float* xl = xm + 2 * BT;                           // [2][BT]
-    xm[g * BT + row] = m_used;
-    xl[g * BT + row] = l;
-    asm volatile("bar.sync 2, 256;" ::: "memory");
-    const float m0 = xm[row], m1 = xm[BT + row];
-    const float M = fmaxf(m0, m1);                     // finite: key 0 is never masked for any row
-    const float f0 = (m0 == -INFINITY) ? 0.f : exp2f(m0 - M);
-    const float f1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - M);
-    const float L = xl[row] * f0 + xl[BT + row] * f1;
     if (ok) {
-      const float a0 = f0 / L, a1 = f1 / L;
+      const float inv = 1.0f / l;
       __nv_bfloat16* orow = out + ((size_t)(tok0 + qpos) * Hq + h) * D;
 #pragma unroll 1
-      for (int c0 = g * 64; c0 < g * 64 + 64; c0 += 32) {   // warpgroup g writes output columns [64g, 64g+64)
-        uint32_t r0[32], r1[32];
+      for (int c0 = 0; c0 < D; c0 += 32) {
+        uint32_t r0[32];
         tmem_ld32(tmem + lane_base + kColO + c0, r0);
-        tmem_ld32(tmem + lane_base + kColO + BT + c0, r1);
         tmem_wait_ld();
         if (qpos < N) {
 #pragma unroll
           for (int c = 0; c < 32; c += 8) {
             float o[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) o[e] = fmaf(__uint_as_float(r1[c + e]), a1, __uint_as_float(r0[c + e]) * a0);
+            for (int e = 0; e < 8; ++e) o[e] = __uint_as_float(r0[c + e]) * inv;
             uint4 w;
             __nv_bfloat162 t0 = __floats2bfloat162_rn(o[0], o[1]), t1 = __floats2bfloat162_rn(o[2], o[3]);
             __nv_bfloat162 t2 = __floats2bfloat162_rn(o[4], o[5]), t3 = __floats2bfloat162_rn(o[6], o[7]);
@@ -482,14 +474,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           }
         }
       }
-      if (g == 0 && qpos < N) lse[(size_t)h * stride + tok0 + qpos] = M + log2f(L);
+      if (qpos < N) lse[(size_t)h * stride + tok0 + qpos] = m_used + log2f(l);
     }
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem, 512);
+    tmem_dealloc(tmem, 256);
   }
 }
 
@@ -512,12 +504,12 @@ EncodeTiledFn encode_fn() {
 }
 
 // [tokens][heads * 128] bf16, boxes of 64 columns x 128 rows, 128-byte swizzle, zero fill out of range.
-bool make_map(CUtensorMap* map, const void* base, int tokens, int heads) {
+bool make_map(CUtensorMap* map, const void* base, int tokens, int heads, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)heads * D, (cuuint64_t)tokens};
   const cuuint64_t strides[1] = {(cuuint64_t)heads * D * 2};
-  const cuuint32_t box[2] = {64, (cuuint32_t)BT};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -529,11 +521,11 @@ bool make_map(CUtensorMap* map, const void* base, int tokens, int heads) {
 cudaError_t buzz_launch_prefill_tc(buzz_ctx* c, const void* q, const void* k, const void* v,
                                    const int32_t* cu, int batch, int total_tokens, int max_seqlen,
                                    void* out, cudaStream_t stream, int* launches) {
-  CUtensorMap mq, mk, mv;
-  if (!make_map(&mq, q, total_tokens, c->sh.q_heads) || !make_map(&mk, k, total_tokens, c->sh.kv_heads) ||
-      !make_map(&mv, v, total_tokens, c->sh.kv_heads))
+  CUtensorMap mq, mk, mk64, mv64;                      // 128-row boxes for Q and pass B's keys, 64-row boxes for pass A's K and V
+  if (!make_map(&mq, q, total_tokens, c->sh.q_heads, BT) || !make_map(&mk, k, total_tokens, c->sh.kv_heads, BT) ||
+      !make_map(&mk64, k, total_tokens, c->sh.kv_heads, KT) || !make_map(&mv64, v, total_tokens, c->sh.kv_heads, KT))
     return cudaErrorInvalidValue;
-  const size_t smemA = sizeof(SmemA), smemB = sizeof(SmemB) + 1024;
+  const size_t smemA = sizeof(SmemA) + 1024, smemB = sizeof(SmemB) + 1024;
   static bool attr_done = false;
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smemA);
@@ -547,7 +539,7 @@ cudaError_t buzz_launch_prefill_tc(buzz_ctx* c, const void* q, const void* k, co
   const int logn = (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0;
   (void)cudaGetLastError();   // drop a stale non-sticky error left by an earlier runtime call of the process
   attn_tc_kernel<<<dim3(tiles, c->sh.q_heads, batch), kThreadsA, smemA, stream>>>(
-      mq, mk, mv, cu, (__nv_bfloat16*)out, c->lse, c->st.status, c->sh.q_heads, c->sh.kv_heads,
+      mq, mk64, mv64, cu, (__nv_bfloat16*)out, c->lse, c->st.status, c->sh.q_heads, c->sh.kv_heads,
       c->sh.max_prompt_tokens, scale_log2, logn);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
