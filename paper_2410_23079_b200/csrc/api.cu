@@ -37,6 +37,10 @@ bool shape_ok(const buzz_shape* s, int budget) {
   return true;
 }
 
+// floats per head of the row-statistics scratch: every sequence may start up to 4 floats later than
+// its token offset (alignment), and a tile read may run 127 rows past a sequence's end
+inline int lse_stride_of(const buzz_shape& s) { return ((s.max_prompt_tokens + 4 * s.max_batch + 128 + 3) & ~3) + 4; }
+
 Layout make_layout(const buzz_shape& s, int budget) {
   Layout L{};
   const size_t e = s.dtype == BUZZ_BF16 ? 2 : 4;
@@ -52,7 +56,7 @@ Layout make_layout(const buzz_shape& s, int budget) {
   L.status = off; off = align_up(off + 4 * sizeof(int32_t));
   L.state_bytes = off;
   off = 0;
-  L.lse = off; off = align_up(off + (size_t)s.q_heads * s.max_prompt_tokens * sizeof(float));
+  L.lse = off; off = align_up(off + (size_t)s.q_heads * lse_stride_of(s) * sizeof(float));
   L.pscore = off; off = align_up(off + (size_t)s.kv_heads * s.max_prompt_tokens * sizeof(float));
   L.stage_q = align_up((size_t)s.max_batch * s.q_heads * s.head_dim * e);
   L.stage_kv = align_up((size_t)s.max_batch * s.kv_heads * s.head_dim * e);
@@ -106,6 +110,7 @@ int buzz_create(buzz_t* out, int sink, int window, int segment, int hitters, int
   c->st.status = reinterpret_cast<int32_t*>(sb + L.status);
   char* sc = static_cast<char*>(scratch_dev);
   c->lse = reinterpret_cast<float*>(sc + L.lse);
+  c->lse_stride = lse_stride_of(*shape);
   c->pscore = reinterpret_cast<float*>(sc + L.pscore);
   c->stage = sc + L.stage;
   c->stage_q = L.stage_q;

@@ -38,7 +38,9 @@ struct buzz_ctx {
   size_t esize;       // bytes per K/V element
   BuzzState st;
   // scratch partition
-  float* lse;         // [q_heads][max_prompt_tokens] row log-sum-exp (log2 domain) of one prefill
+  float* lse;         // [q_heads][lse_stride] row log-sum-exp (log2 domain) of one prefill; the tensor-core path
+                      // starts each sequence's rows at a multiple of four floats (16-byte-aligned bulk copies)
+  int lse_stride;     // floats per head: max_prompt_tokens + 4 per sequence + one tile of slack, a multiple of 4
   float* pscore;      // [kv_heads][max_prompt_tokens] pre-eviction prompt scores
   char* stage;        // staging for the host-buffer entries: per layer q | k | v, then per layer out
   size_t stage_q, stage_kv;  // byte sizes of one q-shaped and one kv-shaped staging tensor

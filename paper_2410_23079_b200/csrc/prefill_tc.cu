@@ -90,11 +90,18 @@ __device__ __forceinline__ void colsum_tile(const uint32_t (&r)[NC], const float
 // shared by two threads, one per compute warpgroup: warpgroup g sums query columns [64g, 64g+64)
 // of every tile, and the two partial sums are added in a fixed order at the end.
 // =================================================================================================
+// A slot of row statistics is rewritten kLseSlots iterations after it was filled. The producer fills
+// the slot of iteration `it` once the MMA of it-2 has completed, which was issued only after every
+// compute thread had taken the logits of it-4 out of TMEM, i.e. had finished iteration it-5.
+constexpr int kLseSlots = 8;
+// Row statistics are stored with each sequence's rows starting at a multiple of four floats, so
+// that a tile's 128 values can be fetched with one 16-byte-aligned bulk copy.
+__device__ __forceinline__ int lse_offset(int tok0, int b) { return (tok0 & ~3) + 4 * b; }
 struct SmemB {
   alignas(1024) unsigned char k[kTileBytes];
   alignas(1024) unsigned char q[2][kTileBytes];
-  float lse[2][8][64];                     // [tile parity][compute warp][column of its half]: per-warp copies,
-  float rs[2][8][64];                      // so the compute warps never meet at a CTA-wide barrier inside the loop
+  alignas(16) float lse[kLseSlots][BT];    // row log-sum-exp of the query tile of iteration it, slot it % kLseSlots (bulk-copied)
+  float rs[2][8][64];                      // log-n row scales, [tile parity][compute warp][column of its half]: per-warp copies
   float part[BT];                          // warpgroup 1's partial column sums
   uint64_t k_full, q_full[2], q_empty[2], s_full[2], s_empty[2];
   uint32_t tmem_base;
@@ -104,7 +111,7 @@ constexpr int kThreadsB = 320;            // TMA warp, MMA warp, 2 x 4 compute w
 __global__ void __launch_bounds__(kThreadsB, 2)
 colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                  const int32_t* __restrict__ cu, const float* __restrict__ lse, float* __restrict__ pscore,
-                 int32_t* status, int Hq, int Hkv, int stride, float scale_log2, int logn) {
+                 int32_t* status, int Hq, int Hkv, int stride, int lse_stride, float scale_log2, int logn) {
   extern __shared__ unsigned char smem_raw[];
   SmemB& sm = *reinterpret_cast<SmemB*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int b = blockIdx.z, kvh = blockIdx.y, G = Hq / Hkv;
@@ -147,8 +154,10 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       for (int it = 0; it < iters; ++it) {
         const int st = it & 1, use = it >> 1;
         if (use > 0 && !mbar_wait(&sm.q_empty[st], (use - 1) & 1)) { tf.raise(1); break; }
-        mbar_expect_tx(&sm.q_full[st], kTileBytes);
+        mbar_expect_tx(&sm.q_full[st], kTileBytes + BT * 4);
         load_tile(sm.q[st], &map_q, (kvh * G + pg) * D, tok0 + pqt * BT, &sm.q_full[st]);
+        bulk_load_1d(sm.lse[it % kLseSlots], lse + (size_t)(kvh * G + pg) * lse_stride + lse_offset(tok0, b) + pqt * BT,
+                     BT * 4, &sm.q_full[st]);
         if (++pqt == q_tiles) { pqt = kt; ++pg; }
       }
     }
@@ -178,31 +187,21 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
     const int kpos = key0 + row;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};           // column c adds into acc[c % 4]: a fixed order
     bool ok = true;
-    // row statistics of tile `it` for this warp's 64 columns (two per lane): fetched from global
-    // memory one iteration ahead, so the load's latency hides behind the previous tile's exponentials
     const int cw = warp - 2;                          // compute warp 0..7
-    // (head of the group, query tile) of an iteration advance together; no divisions in the loop
-    auto fetch_lse = [&](int head, int tile, int e) -> float {
-      const int qpos = tile * BT + g * 64 + lane + 32 * e;
-      return (head < G && qpos < N) ? lse[(size_t)(kvh * G + head) * stride + tok0 + qpos] : 0.f;
-    };
-    int qt = kt, nhead = 0, ntile = kt;                // this iteration's tile; next iteration's (head, tile)
-    float lse_next0 = fetch_lse(0, kt, 0), lse_next1 = fetch_lse(0, kt, 1);
+    int qt = kt, ntile = kt;                          // this iteration's query tile; the next one's
     for (int it = 0; it < iters; ++it) {
       const int st = it & 1, use = it >> 1;
       qt = ntile;
-      if (++ntile == q_tiles) { ntile = kt; ++nhead; }
+      if (++ntile == q_tiles) ntile = kt;
       const int q0 = qt * BT;
-      // this warp's private copy of the tile's row statistics (last read two iterations ago by this warp only)
-      sm.lse[st][cw][lane] = lse_next0;
-      sm.lse[st][cw][lane + 32] = lse_next1;
-      if (logn) {
+      if (logn) {                                     // this warp's private copy of its columns' row scales
         sm.rs[st][cw][lane] = scale_log2 * __logf((float)(q0 + g * 64 + lane + 1)) * kInvLn512;
         sm.rs[st][cw][lane + 32] = scale_log2 * __logf((float)(q0 + g * 64 + lane + 33)) * kInvLn512;
+        __syncwarp();
       }
-      lse_next0 = fetch_lse(nhead, ntile, 0);
-      lse_next1 = fetch_lse(nhead, ntile, 1);
-      __syncwarp();
+      // The tile's row statistics came with its Q tile, on q_full: the MMA thread saw that barrier
+      // complete before it issued the product whose completion s_full reports, so they are in place.
+      // (q_full itself may already be two phases ahead here and must not be waited on.)
       if (!mbar_wait(&sm.s_full[st], use & 1)) { tf.raise(5); ok = false; break; }
       tc_fence_after();
       const bool diag = (qt == kt), tail = (q0 + BT > N);
@@ -216,7 +215,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + st * BT + g * 64 + h * 32, r);
 #pragma unroll
         for (int c = 0; c < 32; c += 4) {
-          const float4 t = *reinterpret_cast<const float4*>(&sm.lse[st][cw][h * 32 + c]);
+          const float4 t = *reinterpret_cast<const float4*>(&sm.lse[it % kLseSlots][g * 64 + h * 32 + c]);
           ls[c] = t.x; ls[c + 1] = t.y; ls[c + 2] = t.z; ls[c + 3] = t.w;
         }
         tmem_wait_ld();
@@ -227,7 +226,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         if (logn) colsum_tile<true, 32>(r, sm.rs[st][cw] + h * 32, ls, scale_log2, diag, tail, q0 + g * 64 + h * 32, kpos, N, acc);
         else colsum_tile<false, 32>(r, sm.rs[st][cw] + h * 32, ls, scale_log2, diag, tail, q0 + g * 64 + h * 32, kpos, N, acc);
       }
-      __syncwarp();                                   // the copy is rewritten two iterations from now
+      if (logn) __syncwarp();                         // the row-scale copy is rewritten two iterations from now
     }
     const float mine = (acc[0] + acc[1]) + (acc[2] + acc[3]);
     if (g == 1) sm.part[row] = mine;
@@ -474,7 +473,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           }
         }
       }
-      if (qpos < N) lse[(size_t)h * stride + tok0 + qpos] = m_used + log2f(l);
+      if (qpos < N) lse[(size_t)h * stride + lse_offset(tok0, b) + qpos] = m_used + log2f(l);
     }
   }
   tc_fence_before();
@@ -540,11 +539,11 @@ cudaError_t buzz_launch_prefill_tc(buzz_ctx* c, const void* q, const void* k, co
   (void)cudaGetLastError();   // drop a stale non-sticky error left by an earlier runtime call of the process
   attn_tc_kernel<<<dim3(tiles, c->sh.q_heads, batch), kThreadsA, smemA, stream>>>(
       mq, mk64, mv64, cu, (__nv_bfloat16*)out, c->lse, c->st.status, c->sh.q_heads, c->sh.kv_heads,
-      c->sh.max_prompt_tokens, scale_log2, logn);
+      c->lse_stride, scale_log2, logn);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   colsum_tc_kernel<<<dim3(tiles, c->sh.kv_heads, batch), kThreadsB, smemB, stream>>>(
-      mq, mk, cu, c->lse, c->pscore, c->st.status, c->sh.q_heads, c->sh.kv_heads, c->sh.max_prompt_tokens,
+      mq, mk, cu, c->lse, c->pscore, c->st.status, c->sh.q_heads, c->sh.kv_heads, c->sh.max_prompt_tokens, c->lse_stride,
       scale_log2, logn);
   *launches += 2;
   return cudaGetLastError();
