@@ -103,7 +103,7 @@ struct SmemB {
   alignas(16) float lse[kLseSlots][BT];    // row log-sum-exp of the query tile of iteration it, slot it % kLseSlots (bulk-copied)
   float rs[2][8][64];                      // log-n row scales, [tile parity][compute warp][column of its half]: per-warp copies
   float part[BT];                          // warpgroup 1's partial column sums
-  uint64_t k_full, q_full[2], q_empty[2], s_full[2], s_empty[2];
+  uint64_t k_full, q_full[2], q_empty[2], s_full[2], s_empty[2], lse_full[kLseSlots];
   uint32_t tmem_base;
 };
 
@@ -132,6 +132,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       mbar_init(&sm.s_full[s], 1);
       mbar_init(&sm.s_empty[s], 256);
     }
+    for (int s = 0; s < kLseSlots; ++s) mbar_init(&sm.lse_full[s], 1);
     fence_barrier_init();
   }
   if (warp == 1) {
@@ -154,10 +155,13 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
       for (int it = 0; it < iters; ++it) {
         const int st = it & 1, use = it >> 1;
         if (use > 0 && !mbar_wait(&sm.q_empty[st], (use - 1) & 1)) { tf.raise(1); break; }
-        mbar_expect_tx(&sm.q_full[st], kTileBytes + BT * 4);
+        mbar_expect_tx(&sm.q_full[st], kTileBytes);
         load_tile(sm.q[st], &map_q, (kvh * G + pg) * D, tok0 + pqt * BT, &sm.q_full[st]);
+        // the tile's row statistics: a barrier of their own, because the threads that read them must
+        // observe the copy's completion themselves (q_full may be two phases ahead by then)
+        mbar_expect_tx(&sm.lse_full[it % kLseSlots], BT * 4);
         bulk_load_1d(sm.lse[it % kLseSlots], lse + (size_t)(kvh * G + pg) * lse_stride + lse_offset(tok0, b) + pqt * BT,
-                     BT * 4, &sm.q_full[st]);
+                     BT * 4, &sm.lse_full[it % kLseSlots]);
         if (++pqt == q_tiles) { pqt = kt; ++pg; }
       }
     }
@@ -199,9 +203,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
         sm.rs[st][cw][lane + 32] = scale_log2 * __logf((float)(q0 + g * 64 + lane + 33)) * kInvLn512;
         __syncwarp();
       }
-      // The tile's row statistics came with its Q tile, on q_full: the MMA thread saw that barrier
-      // complete before it issued the product whose completion s_full reports, so they are in place.
-      // (q_full itself may already be two phases ahead here and must not be waited on.)
+      if (!mbar_wait(&sm.lse_full[it % kLseSlots], (it / kLseSlots) & 1)) { tf.raise(6); ok = false; break; }
       if (!mbar_wait(&sm.s_full[st], use & 1)) { tf.raise(5); ok = false; break; }
       tc_fence_after();
       const bool diag = (qt == kt), tail = (q0 + BT > N);
@@ -219,6 +221,7 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
           ls[c] = t.x; ls[c + 1] = t.y; ls[c + 2] = t.z; ls[c + 3] = t.w;
         }
         tmem_wait_ld();
+        tmem_pin32(r);
         if (h == 1) {
           tc_fence_before();
           mbar_arrive(&sm.s_empty[st]);                // S^T[st] may be overwritten once all 256 have arrived
@@ -390,21 +393,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       if (!mbar_wait(&sm.s_full[sb], (j >> 1) & 1)) { tf.raise(17); ok = false; break; }
       tc_fence_after();
       // the raw logits of this row (rs > 0, so the maximum can be taken before scaling)
-      float s[64];
-      tmem_ld32(tmem + lane_base + colS, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-      tmem_ld32(tmem + lane_base + colS + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+      uint32_t sa[32], sb2[32];
+      tmem_ld32(tmem + lane_base + colS, sa);
+      tmem_ld32(tmem + lane_base + colS + 32, sb2);
       tmem_wait_ld();
+      tmem_pin32(sa);
+      tmem_pin32(sb2);
+      float s[64];
+#pragma unroll
+      for (int c = 0; c < 32; ++c) { s[c] = __uint_as_float(sa[c]); s[32 + c] = __uint_as_float(sb2[c]); }
       if (j * KT + KT - 1 > row0) {                    // a tile that crosses the diagonal: causal mask
 #pragma unroll
         for (int c = 0; c < 64; ++c)
           if (j * KT + c > qpos) s[c] = -INFINITY;
       }
-      float mx4[4] = {s[0], s[1], s[2], s[3]};         // four chains of three-input maxima
+      float mx4[4] = {s[0], s[1], s[2], s[3]};         // four chains of three-input maxima over s[4..63]
 #pragma unroll
-      for (int c = 4; c < 64; c += 8) {
+      for (int c = 4; c + 8 <= 64; c += 8) {           // s[4..59]
 #pragma unroll
         for (int e = 0; e < 4; ++e) mx4[e] = max3(mx4[e], s[c + 2 * e], s[c + 2 * e + 1]);
       }
+      mx4[0] = max3(mx4[0], s[60], s[61]);
+      mx4[1] = max3(mx4[1], s[62], s[63]);
       const float mx = fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]) * rs;   // -inf if the whole tile is masked for this row
       const float m_new = fmaxf(m_used, mx);
       if (j == 0) {
@@ -422,6 +432,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             uint32_t r[32];
             tmem_ld32(tmem + lane_base + kColO + c0, r);
             tmem_wait_ld();
+            tmem_pin32(r);
 #pragma unroll
             for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
             tmem_st32(tmem + lane_base + kColO + c0, r);
@@ -458,6 +469,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         uint32_t r0[32];
         tmem_ld32(tmem + lane_base + kColO + c0, r0);
         tmem_wait_ld();
+        tmem_pin32(r0);
         if (qpos < N) {
 #pragma unroll
           for (int c = 0; c < 32; c += 8) {
