@@ -5,19 +5,19 @@
 //   O = Softmax(Q K^T / sqrt(d)) V, causal, per sequence and query head, and for every key j
 //   score_j = sum over the group's query heads and rows i >= j of P_ij.
 // The column sums need each row's FINAL normaliser, so S = Q K^T is formed twice:
-//   pass A  (attn_tc_kernel, query-tile stationary) flash-style attention: S in TMEM, one thread
-//           per row does the online softmax, P goes back to TMEM as bf16 and is the A operand of
-//           the P V MMA; the output accumulators live in TMEM and are rescaled lazily (only when a
-//           row maximum grows by more than 2^8). Each row is shared by two threads (one per softmax
-//           warpgroup, half the key columns and an accumulator each). Writes O and the row
-//           log2-sum-exp.
+//   pass A  (attn_tc_kernel, query-tile stationary) flash-style attention over key tiles of 64: S
+//           in TMEM, one thread per row does the online softmax, P goes back to TMEM as bf16 and is
+//           the A operand of the P V MMA; the output accumulator lives in TMEM and is rescaled
+//           lazily (only when a row maximum grows by more than 2^20). Two CTAs share an SM.
+//           Writes O and the row log2-sum-exp.
 //   pass B  (colsum_tc_kernel, key-tile stationary) S^T = K Q^T in TMEM with KEYS on the TMEM
 //           lanes, so one thread owns one key: it forms the exact probabilities 2^(S - lse) in
 //           fp32 and adds them up over the query rows in a fixed order (heads, then tiles, then
 //           rows ascending) -- no cross-thread reduction, no atomics, bit-reproducible.
-// Warp roles in both kernels: warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM owner),
-// the remaining warps = one thread per TMEM lane (per warpgroup). All mbarrier waits are bounded; a wait that gives up sets
-// BUZZ_ERR_TIMEOUT and the CTA runs to its end without touching more data.
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (and TMEM owner; in pass A a further warp
+// issues the second product), the remaining warps = one thread per TMEM lane. All mbarrier waits
+// are bounded; a wait that gives up sets BUZZ_ERR_TIMEOUT and the CTA runs to its end without
+// touching more data.
 #include <math.h>
 
 #include "buzz_internal.cuh"
