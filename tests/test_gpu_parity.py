@@ -405,3 +405,55 @@ def test_decode_layers_rejects_bad_layer_lists(cuda_device):
     with pytest.raises(BuzzError):
         bz.decode_layers_host([1, 1], qd[0].cpu(), o.cpu())
     bz.close()
+
+
+@pytest.mark.gpu
+def test_step_replayed_from_a_cuda_graph(cuda_device):
+    """One decode step of a layer stack plus the eviction call, captured once in a CUDA graph and
+    replayed with fresh inputs in static buffers, leaves the same outputs and caches as direct calls
+    (evictions included: the trigger is a device predicate, so the captured launches need no host
+    decision)."""
+    w = workloads.scaled(workloads.get("C4"), layers=3, batch=2, q_heads=8, kv_heads=2, prompt_min=150,
+                         prompt_max=150, decode_steps=45, window=32, budget=180)
+    pre, dec = _stack(w)
+    ref, cap = make_buzz(w), make_buzz(w)
+    for bz in (ref, cap):
+        for l in range(w.layers):
+            q, k, v, cu = pre[l]
+            bz.prefill(l, q, k, v, cu, 150, torch.empty_like(q))
+    L = list(range(w.layers))
+    sq = [torch.empty_like(dec[l][0][0]) for l in L]
+    sk = [torch.empty_like(dec[l][1][0]) for l in L]
+    sv = [torch.empty_like(dec[l][2][0]) for l in L]
+    so = [torch.empty_like(dec[l][0][0]) for l in L]
+
+    def load(t):
+        for l in L:
+            sq[l].copy_(dec[l][0][t]); sk[l].copy_(dec[l][1][t]); sv[l].copy_(dec[l][2][t])
+
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    load(0)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):        # step 0 is only recorded here, not run
+            cap.decode_layers(L, sq, sk, sv, so, stream=side)
+            cap.evict(-1, stream=side)
+    torch.cuda.synchronize()
+    for t in range(w.decode_steps):
+        o_ref = [torch.empty_like(so[l]) for l in L]
+        ref.decode_layers(L, [dec[l][0][t] for l in L], [dec[l][1][t] for l in L], [dec[l][2][t] for l in L], o_ref)
+        ref.evict(-1)
+        load(t)
+        graph.replay()
+        torch.cuda.synchronize()
+        for l in L:
+            assert torch.equal(so[l], o_ref[l]), f"step {t} layer {l}"
+    for l in L:
+        for b in range(w.batch):
+            a, c = ref.export_state(l, b, 1), cap.export_state(l, b, 1)
+            assert (a["n"], a["n_old"], a["total_len"]) == (c["n"], c["n_old"], c["total_len"])
+            assert torch.equal(a["pos"], c["pos"]) and torch.equal(a["score"], c["score"]) and torch.equal(a["k"], c["k"])
+    assert ref.export_state(0, 0, 0)["n"] < 150 + w.decode_steps      # evictions happened on the way
+    assert ref.status() == 0 and cap.status() == 0
+    ref.close(); cap.close()
