@@ -86,6 +86,12 @@ def _after_evict(n, n_old, w):
     return w.sink + m + w.window, m, True
 
 
+def _workload_name(w) -> str:
+    return (f"{w.name}: {w.layers} layers x {w.batch} seqs x {w.q_heads}/{w.kv_heads} heads, d={w.head_dim}, "
+            f"prompt {w.prompt_min}..{w.prompt_max}, sink {w.sink} window {w.window} segment {w.segment} "
+            f"hitters {w.hitters} budget {w.budget}")
+
+
 def max_over_ranks(value: float, dist, device) -> float:
     """Slowest rank's time: every multi-GPU number is the max over ranks (replicas run independently)."""
     if dist is None:
@@ -346,9 +352,7 @@ def run_ours(args):
     line = dict(metric="decode tokens/s (attention + BUZZ eviction)", value=whole_job_rate(w.batch * K, world, ms),
                 unit="tokens/s", n_gpus=world, steps=K, warmup=W, ms_per_step=ms / K, higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype=w.dtype, data="synthetic",
-                config=dict(workload=f"{w.name}: {w.layers} layers x {w.batch} seqs x {w.q_heads}/{w.kv_heads} heads, d={w.head_dim}, "
-                                     f"prompt {w.prompt_min}..{w.prompt_max}, sink {w.sink} window {w.window} segment {w.segment} "
-                                     f"hitters {w.hitters} budget {w.budget}",
+                config=dict(workload=_workload_name(w),
                             parallelism="replicas only" if world > 1 else "single GPU",
                             l2="per-step K/V working set (GBs) exceeds the 126 MB L2; no flush needed",
                             decode_input_pool=pool, evictions_in_timed_region=timed_evictions),
@@ -421,7 +425,7 @@ def run_reference(args):
                 n_gpus=int(os.environ.get("WORLD_SIZE", 1)), steps=args.steps, warmup=args.warmup,
                 ms_per_step=1e3 * w.batch / v, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="f64", data="synthetic",
-                config=dict(workload=f"{w.name} (bounded sample per step, see cpu_baseline.sample)"),
+                config=dict(workload=_workload_name(w), sample="each step is a bounded sample of this workload, see cpu_baseline.sample"),
                 cpu_baseline=base, e2e=dict(value=v, unit="tokens/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0),
                 gpu_launches=0)
     print(json.dumps(line))
