@@ -133,7 +133,9 @@ int buzz_decode_step(buzz_t ctx, int layer, const void* q, const void* k_new, co
  * library's staging area in scratch, runs the step, copies `out` back, all on `stream`, without
  * synchronising. Layouts as in buzz_decode_step. If the three inputs are contiguous in host memory in
  * the order q, k_new, v_new (one allocation holding the packed record) they are sent in a single
- * copy; buffers that merely happen to be adjacent but were pinned separately are copied one by one. */
+ * copy; buffers that merely happen to be adjacent but were pinned separately are copied one by one.
+ * If all four buffers are pinned and mapped, the kernel reads and writes them in place and nothing
+ * is copied (see buzz_decode_layers_host). */
 int buzz_decode_step_host(buzz_t ctx, int layer, const void* q_host, const void* k_new_host,
                           const void* v_new_host, void* out_host, void* stream);
 
@@ -155,8 +157,12 @@ int buzz_decode_layers(buzz_t ctx, int count, const int* layers, const void* con
 
 /* buzz_decode_layers with HOST buffers (pinned memory recommended). `in_host` is one packed buffer,
  * for each listed layer in order its q | k_new | v_new tensors (layouts of buzz_decode_step, sized by
- * that layer's batch); `out_host` receives the outputs packed the same way. One host-to-device
- * copy, the launches, one device-to-host copy, all on `stream`, without synchronising. */
+ * that layer's batch); `out_host` receives the outputs packed the same way. Nothing synchronises.
+ * Buffers the GPU can address in place (pinned and mapped: cudaHostAlloc, cudaHostRegister, a
+ * framework's pinned tensors) are read and written by the kernels directly, so the transfers overlap
+ * the step; otherwise: one host-to-device copy into the library's staging area, the launches, one
+ * device-to-host copy, all on `stream`. Either way `out_host` is valid once `stream` has reached the
+ * end of the call, and `in_host` must stay unchanged until then. */
 int buzz_decode_layers_host(buzz_t ctx, int count, const int* layers, const void* in_host,
                             void* out_host, void* stream);
 

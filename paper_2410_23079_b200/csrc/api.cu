@@ -67,6 +67,23 @@ Layout make_layout(const buzz_shape& s, int budget) {
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The device-side address of a HOST buffer the GPU can read and write in place (pinned and mapped,
+// which is what cudaHostAlloc / cudaHostRegister give under unified addressing), or null if the
+// buffer is pageable, partly outside one such allocation, or misaligned for the kernels.
+void* mapped_device_ptr(const void* host, size_t bytes) {
+  if (!host || bytes == 0) return nullptr;
+  cudaPointerAttributes first, last;
+  if (cudaPointerGetAttributes(&first, host) != cudaSuccess ||
+      cudaPointerGetAttributes(&last, static_cast<const char*>(host) + bytes - 1) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return nullptr;
+  }
+  if (first.type != cudaMemoryTypeHost || last.type != cudaMemoryTypeHost || !first.devicePointer || !last.devicePointer)
+    return nullptr;
+  if (static_cast<char*>(last.devicePointer) - static_cast<char*>(first.devicePointer) != (ptrdiff_t)(bytes - 1)) return nullptr;
+  return aligned16(first.devicePointer) ? first.devicePointer : nullptr;
+}
+
 }  // namespace
 
 extern "C" {
@@ -176,6 +193,14 @@ int buzz_decode_step_host(buzz_t c, int layer, const void* q_host, const void* k
   const size_t kb = (size_t)batch * c->sh.kv_heads * c->sh.head_dim * c->esize;
   // staging is packed q | k | v (row sizes are multiples of 16 bytes), so host buffers laid out the
   // same way go down in ONE copy; `out` has its own region behind them
+  {   // buffers the GPU can address in place need no staging copies: the kernel reads and writes them over the bus
+    void* mq = mapped_device_ptr(q_host, qb);
+    void* mk = mapped_device_ptr(k_new_host, kb);
+    void* mv = mapped_device_ptr(v_new_host, kb);
+    void* mo = mapped_device_ptr(out_host, qb);
+    if (mq && mk && mv && mo)
+      return buzz_launch_decode(c, layer, mq, mk, mv, mo, s) == cudaSuccess ? BUZZ_OK : BUZZ_ERR_CUDA;
+  }
   char* dq = c->stage;
   char* dk = dq + qb;
   char* dv = dk + kb;
@@ -247,7 +272,18 @@ int buzz_decode_layers_host(buzz_t c, int count, const int* layers, const void* 
   if (in_bytes == 0) return BUZZ_OK;
   char* din = c->stage;
   char* dout = c->stage + (size_t)c->sh.layers * (c->stage_q + 2 * c->stage_kv);
-  if (cudaMemcpyAsync(din, in_host, in_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+  // Pinned, mapped host buffers are used in place: each kernel fetches its few input rows and writes
+  // its output rows over the bus while the cache streams from HBM, so the transfers overlap the
+  // step instead of bracketing it. Pageable buffers go through the staging area with one copy each way.
+  void* min = mapped_device_ptr(in_host, in_bytes);
+  void* mout = mapped_device_ptr(out_host, out_bytes);
+  const bool in_place = min && mout;
+  if (in_place) {
+    din = static_cast<char*>(min);
+    dout = static_cast<char*>(mout);
+  } else if (cudaMemcpyAsync(din, in_host, in_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+    return BUZZ_ERR_CUDA;
+  }
   size_t io = 0, oo = 0;
   int pos = 0;
   for (int i = 0; i < count; ++i) {
@@ -263,7 +299,7 @@ int buzz_decode_layers_host(buzz_t c, int count, const int* layers, const void* 
     oo += b * row_q;
     ++pos;
   }
-  if (cudaMemcpyAsync(out_host, dout, out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (!in_place && cudaMemcpyAsync(out_host, dout, out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return BUZZ_ERR_CUDA;
   return BUZZ_OK;
 }
 

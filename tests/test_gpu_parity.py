@@ -283,8 +283,8 @@ def test_decode_step_host_matches_device_entry(cuda_device):
                          prompt_max=260, decode_steps=6, window=32, budget=300)
     q, k, v, cu = workloads.prefill_inputs(w, 0, "cuda:0")
     qd, kd, vd = workloads.decode_inputs(w, 0, "cuda:0")
-    ref, sep, packed = make_buzz(w), make_buzz(w), make_buzz(w)
-    for bz in (ref, sep, packed):
+    ref, sep, packed, paged = make_buzz(w), make_buzz(w), make_buzz(w), make_buzz(w)
+    for bz in (ref, sep, packed, paged):
         bz.prefill(0, q, k, v, cu, 260, torch.empty_like(q))
     nq, nk = qd[0].numel(), kd[0].numel()
     for t in range(w.decode_steps):
@@ -296,14 +296,17 @@ def test_decode_step_host_matches_device_entry(cuda_device):
         rec = torch.cat([hq.reshape(-1), hk.reshape(-1), hv.reshape(-1)]).pin_memory()
         o_pk = torch.empty_like(hq).pin_memory()
         packed.decode_step_host(0, rec[:nq], rec[nq:nq + nk], rec[nq + nk:], o_pk)
+        rec_p = torch.empty(rec.shape, dtype=rec.dtype).copy_(rec)      # pageable memory: staged copies
+        o_pg = torch.empty(hq.shape, dtype=hq.dtype)
+        paged.decode_step_host(0, rec_p[:nq], rec_p[nq:nq + nk], rec_p[nq + nk:], o_pg)
         torch.cuda.synchronize()
-        assert torch.equal(o_sep, o_ref.cpu()) and torch.equal(o_pk, o_ref.cpu())
-    for bz in (sep, packed):
+        assert torch.equal(o_sep, o_ref.cpu()) and torch.equal(o_pk, o_ref.cpu()) and torch.equal(o_pg, o_ref.cpu())
+    for bz in (sep, packed, paged):
         for b in range(2):
             a, c = ref.export_state(0, b, 1), bz.export_state(0, b, 1)
             assert a["n"] == c["n"] and torch.equal(a["score"], c["score"]) and torch.equal(a["k"], c["k"])
         assert bz.status() == 0
-    for bz in (ref, sep, packed):
+    for bz in (ref, sep, packed, paged):
         bz.close()
 
 
@@ -323,8 +326,8 @@ def test_decode_layers_matches_single_layer_calls(cuda_device, shape):
     w = workloads.scaled(workloads.get("C4"), layers=4, prompt_min=150, prompt_max=150, decode_steps=40,
                          window=32, budget=180, **shape)
     pre, dec = _stack(w)
-    ref, multi, host = make_buzz(w), make_buzz(w), make_buzz(w)
-    for bz in (ref, multi, host):
+    ref, multi, host, paged = make_buzz(w), make_buzz(w), make_buzz(w), make_buzz(w)
+    for bz in (ref, multi, host, paged):
         for l in range(w.layers):
             q, k, v, cu = pre[l]
             bz.prefill(l, q, k, v, cu, 150, torch.empty_like(q))
@@ -339,15 +342,20 @@ def test_decode_layers_matches_single_layer_calls(cuda_device, shape):
                             [dec[l][2][t] for l in order], [o_m[l] for l in order])
         rec = torch.cat([torch.cat([dec[l][i][t].reshape(-1) for i in range(3)]) for l in order]).cpu().pin_memory()
         o_h = torch.empty(sum(o_ref[l].numel() for l in order), dtype=rec.dtype).pin_memory()
-        host.decode_layers_host(order, rec, o_h)
+        host.decode_layers_host(order, rec, o_h)          # pinned: read and written in place by the kernels
+        rec_p = torch.empty(rec.shape, dtype=rec.dtype).copy_(rec)      # pageable: through the staging area
+        o_p = torch.empty(o_h.shape, dtype=o_h.dtype)
+        assert not rec_p.is_pinned() and not o_p.is_pinned()
+        paged.decode_layers_host(order, rec_p, o_p)
         if t % 2 == 0 or t >= 20:            # early odd steps: the next call follows the last one directly
-            for bz in (ref, multi, host):
+            for bz in (ref, multi, host, paged):
                 bz.evict(-1)
         torch.cuda.synchronize()
         flat = torch.cat([o_ref[l].reshape(-1) for l in order]).cpu()
         assert torch.equal(torch.cat([o_m[l].reshape(-1) for l in order]).cpu(), flat), f"step {t}"
-        assert torch.equal(o_h, flat), f"host entry, step {t}"
-    for bz in (multi, host):
+        assert torch.equal(o_h, flat), f"host entry, pinned buffers, step {t}"
+        assert torch.equal(o_p, flat), f"host entry, pageable buffers, step {t}"
+    for bz in (multi, host, paged):
         for l in range(w.layers):
             for b in range(w.batch):
                 a, c = ref.export_state(l, b, w.kv_heads - 1), bz.export_state(l, b, w.kv_heads - 1)
@@ -355,7 +363,7 @@ def test_decode_layers_matches_single_layer_calls(cuda_device, shape):
                 assert torch.equal(a["pos"], c["pos"]) and torch.equal(a["score"], c["score"])
                 assert torch.equal(a["k"], c["k"]) and torch.equal(a["v"], c["v"])
         assert bz.status() == 0
-    for bz in (ref, multi, host):
+    for bz in (ref, multi, host, paged):
         bz.close()
 
 
