@@ -276,6 +276,7 @@ struct SmemA {
 constexpr uint32_t kColO = 128;
 constexpr float kRescaleThreshold = 20.0f;    // log2: rescale O only when a row max grows by > 2^20
                                               // (P, the row sums and O stay far inside the fp32/bf16 exponent range)
+constexpr float kSpeculationLimit = 1048576.0f;   // 2^kRescaleThreshold
 
 // K-major [64 keys][128 dims] tile as two swizzled blocks: descriptor of k-step ks (16 dims).
 __device__ __forceinline__ uint64_t kmajor_desc_kv(uint32_t tile_saddr, int ks) {
@@ -407,53 +408,71 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         for (int c = 0; c < 64; ++c)
           if (j * KT + c > qpos) s[c] = -INFINITY;
       }
-      float mx4[4] = {s[0], s[1], s[2], s[3]};         // four chains of three-input maxima over s[4..63]
-#pragma unroll
-      for (int c = 4; c + 8 <= 64; c += 8) {           // s[4..59]
-#pragma unroll
-        for (int e = 0; e < 4; ++e) mx4[e] = max3(mx4[e], s[c + 2 * e], s[c + 2 * e + 1]);
-      }
-      mx4[0] = max3(mx4[0], s[60], s[61]);
-      mx4[1] = max3(mx4[1], s[62], s[63]);
-      const float mx = fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]) * rs;   // -inf if the whole tile is masked for this row
-      const float m_new = fmaxf(m_used, mx);
-      if (j == 0) {
-        m_used = m_new;                                // finite: key 0 is never masked
-      } else {
-        const bool need = m_new > m_used + kRescaleThreshold;
-        if (__any_sync(0xffffffffu, need)) {
-          const float alpha = need ? exp2f(m_used - m_new) : 1.0f;
-          if (need) m_used = m_new;
-          l *= alpha;
-          if (!mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
-          tc_fence_after();
-#pragma unroll 1
-          for (int c0 = 0; c0 < D; c0 += 32) {
-            uint32_t r[32];
-            tmem_ld32(tmem + lane_base + kColO + c0, r);
-            tmem_wait_ld();
-            tmem_pin32(r);
-#pragma unroll
-            for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
-            tmem_st32(tmem + lane_base + kColO + c0, r);
-          }
-          tmem_wait_st();
-        }
-      }
-      // P = 2^(S rs - m) as bf16 pairs over the first 32 columns of this S buffer (S is in registers)
-      const float neg_m = -m_used;
-      float l4[4] = {0.f, 0.f, 0.f, 0.f};
+      // P = 2^(S rs - m) as bf16 pairs (they will overwrite the first 32 columns of this S buffer) and their sum
       uint32_t pk[32];
+      float tile_sum = 0.f;
+      auto exp_pass = [&]() {
+        const float neg_m = -m_used;
+        float l4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c = 0; c < 32; ++c) {
-        const float p0 = exp2f(fmaf(s[2 * c], rs, neg_m));
-        const float p1 = exp2f(fmaf(s[2 * c + 1], rs, neg_m));
-        l4[c & 3] += p0 + p1;
-        const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
-        pk[c] = *reinterpret_cast<const uint32_t*>(&pp);
+        for (int c = 0; c < 32; ++c) {
+          const float p0 = exp2f(fmaf(s[2 * c], rs, neg_m));
+          const float p1 = exp2f(fmaf(s[2 * c + 1], rs, neg_m));
+          l4[c & 3] += p0 + p1;
+          const __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1);
+          pk[c] = *reinterpret_cast<const uint32_t*>(&pp);
+        }
+        tile_sum = (l4[0] + l4[1]) + (l4[2] + l4[3]);
+      };
+      // After the first tile the maximum in use is almost always good enough (O is only rescaled when
+      // a row maximum grows by more than 2^kRescaleThreshold), so P is formed SPECULATIVELY with it and
+      // the pass over the logits that takes their maximum is skipped: if the tile's probabilities add
+      // up to no more than 2^kRescaleThreshold, none of them exceeds it and the tile stands. Otherwise
+      // (some row of the warp says so, or an overflow made the sum infinite) the maximum is taken
+      // properly, O is rescaled where needed and P is formed again.
+      bool settled = false;
+      if (j > 0) {
+        exp_pass();
+        settled = !__any_sync(0xffffffffu, !(tile_sum <= kSpeculationLimit));
+      }
+      if (!settled) {
+        float mx4[4] = {s[0], s[1], s[2], s[3]};       // four chains of three-input maxima over s[4..63]
+#pragma unroll
+        for (int c = 4; c + 8 <= 64; c += 8) {         // s[4..59]
+#pragma unroll
+          for (int e = 0; e < 4; ++e) mx4[e] = max3(mx4[e], s[c + 2 * e], s[c + 2 * e + 1]);
+        }
+        mx4[0] = max3(mx4[0], s[60], s[61]);
+        mx4[1] = max3(mx4[1], s[62], s[63]);
+        const float mx = fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]) * rs;   // -inf if the whole tile is masked for this row
+        const float m_new = fmaxf(m_used, mx);
+        if (j == 0) {
+          m_used = m_new;                              // finite: key 0 is never masked
+        } else {
+          const bool need = m_new > m_used + kRescaleThreshold;
+          if (__any_sync(0xffffffffu, need)) {
+            const float alpha = need ? exp2f(m_used - m_new) : 1.0f;
+            if (need) m_used = m_new;
+            l *= alpha;
+            if (!mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
+            tc_fence_after();
+#pragma unroll 1
+            for (int c0 = 0; c0 < D; c0 += 32) {
+              uint32_t r[32];
+              tmem_ld32(tmem + lane_base + kColO + c0, r);
+              tmem_wait_ld();
+              tmem_pin32(r);
+#pragma unroll
+              for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
+              tmem_st32(tmem + lane_base + kColO + c0, r);
+            }
+            tmem_wait_st();
+          }
+        }
+        exp_pass();
       }
       tmem_st32(tmem + lane_base + colS, pk);
-      l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
+      l += tile_sum;
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&sm.p_full[sb]);
