@@ -8,7 +8,8 @@
 //   pass A  (attn_tc_kernel, query-tile stationary) flash-style attention over key tiles of 64: S
 //           in TMEM, one thread per row does the online softmax, P goes back to TMEM as bf16 and is
 //           the A operand of the P V MMA; the output accumulator lives in TMEM and is rescaled
-//           lazily (only when a row maximum grows by more than 2^20). Two CTAs share an SM.
+//           lazily (P is formed with the maximum in use; only a tile whose probabilities add up
+//           to more than 2^20 makes the warp take maxima and rescale). Two CTAs share an SM.
 //           Writes O and the row log2-sum-exp.
 //   pass B  (colsum_tc_kernel, key-tile stationary) S^T = K Q^T in TMEM with KEYS on the TMEM
 //           lanes, so one thread owns one key: it forms the exact probabilities 2^(S - lse) in
@@ -274,9 +275,12 @@ struct SmemA {
   uint32_t tmem_base;
 };
 constexpr uint32_t kColO = 128;
-constexpr float kRescaleThreshold = 20.0f;    // log2: rescale O only when a row max grows by > 2^20
-                                              // (P, the row sums and O stay far inside the fp32/bf16 exponent range)
-constexpr float kSpeculationLimit = 1048576.0f;   // 2^kRescaleThreshold
+// A speculative tile stands while its probabilities add up to at most 2^20 (P, the row sums and O stay
+// far inside the fp32/bf16 exponent range). When one does not, every row of the warp whose maximum
+// has grown by more than 2^8 since it was last set is brought up to date, so that a row is not
+// caught again at the next tile.
+constexpr float kRescaleThreshold = 8.0f;
+constexpr float kSpeculationLimit = 1048576.0f;
 
 // K-major [64 keys][128 dims] tile as two swizzled blocks: descriptor of k-step ks (16 dims).
 __device__ __forceinline__ uint64_t kmajor_desc_kv(uint32_t tile_saddr, int ks) {
@@ -424,10 +428,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
         tile_sum = (l4[0] + l4[1]) + (l4[2] + l4[3]);
       };
-      // After the first tile the maximum in use is almost always good enough (O is only rescaled when
-      // a row maximum grows by more than 2^kRescaleThreshold), so P is formed SPECULATIVELY with it and
+      // After the first tile the maximum in use is almost always good enough (a stale maximum only
+      // makes P, the row sum and O larger by the same factor), so P is formed SPECULATIVELY with it and
       // the pass over the logits that takes their maximum is skipped: if the tile's probabilities add
-      // up to no more than 2^kRescaleThreshold, none of them exceeds it and the tile stands. Otherwise
+      // up to no more than kSpeculationLimit, none of them exceeds it and the tile stands. Otherwise
       // (some row of the warp says so, or an overflow made the sum infinite) the maximum is taken
       // properly, O is rescaled where needed and P is formed again.
       bool settled = false;
