@@ -119,6 +119,7 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   const int tot = st.total[inst];
   if (n0 >= pol.budget) {          // uniform over the cluster: every CTA read the same n0
     if (rank == 0 && tid == 0) buzz_set_status(st.status, BUZZ_ERR_OVERFLOW, (int)inst, n0);
+    if (mode == kOverlap) asm volatile("griddepcontrol.wait;" ::: "memory");   // still finish after the member before
     return;
   }
   const int n1 = n0 + 1;

@@ -465,3 +465,39 @@ def test_step_replayed_from_a_cuda_graph(cuda_device):
     assert ref.export_state(0, 0, 0)["n"] < 150 + w.decode_steps      # evictions happened on the way
     assert ref.status() == 0 and cap.status() == 0
     ref.close(); cap.close()
+
+
+@pytest.mark.gpu
+def test_decode_layers_with_uneven_and_empty_layers(cuda_device):
+    """Layers prefilled with different batch sizes, and a layer that was never prefilled, in one
+    multi-layer call: each layer steps its own sequences, the empty one launches nothing; a full
+    cache inside the call is reported and skipped like in a single-layer call."""
+    w = workloads.scaled(workloads.get("C4"), layers=3, batch=3, q_heads=8, kv_heads=2, prompt_min=120,
+                         prompt_max=120, decode_steps=8, window=16, budget=124)
+    pre, dec = _stack(w)
+    ref, multi = make_buzz(w), make_buzz(w)
+    nb = {0: 3, 1: 0, 2: 2}                                    # sequences per layer (layer 1 stays empty)
+    for bz in (ref, multi):
+        for l, b in nb.items():
+            if b:
+                q, k, v, cu = pre[l]
+                bz.prefill(l, q[:b * 120], k[:b * 120], v[:b * 120], cu[:b + 1], 120, torch.empty_like(q[:b * 120]))
+    for t in range(w.decode_steps):
+        o_ref = {l: torch.zeros_like(dec[l][0][t]) for l in nb}
+        o_m = {l: torch.zeros_like(dec[l][0][t]) for l in nb}
+        for l, b in nb.items():
+            if b:
+                ref.decode_step(l, dec[l][0][t][:b], dec[l][1][t][:b], dec[l][2][t][:b], o_ref[l][:b])
+        L = [2, 1, 0]
+        multi.decode_layers(L, [dec[l][0][t][:max(nb[l], 1)] for l in L], [dec[l][1][t][:max(nb[l], 1)] for l in L],
+                            [dec[l][2][t][:max(nb[l], 1)] for l in L], [o_m[l][:max(nb[l], 1)] for l in L])
+        torch.cuda.synchronize()
+        for l in nb:
+            assert torch.equal(o_ref[l], o_m[l]), f"step {t} layer {l}"
+    # 120 + 8 steps against a budget of 124 and no eviction call: the last steps found the caches full
+    assert ref.status() == -2 and multi.status() == -2          # BUZZ_ERR_OVERFLOW
+    for l, b in nb.items():
+        for s in range(b):
+            a, c = ref.export_state(l, s, 0), multi.export_state(l, s, 0)
+            assert a["n"] == c["n"] == 124 and torch.equal(a["score"], c["score"]) and torch.equal(a["k"], c["k"])
+    ref.close(); multi.close()
