@@ -262,14 +262,14 @@ colsum_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constan
 constexpr int KT = 64;                    // keys per tile in pass A
 constexpr uint32_t kKvBlockBytes = KT * 128;        // one [64 keys x 64 bf16] swizzled block
 constexpr uint32_t kKvTileBytes = 2 * kKvBlockBytes;
-constexpr int kThreadsA = 352;            // TMA warp, Q K^T issuer, 2 x 4 softmax warps, P V issuer
+constexpr int kThreadsA = 224;            // TMA warp, Q K^T issuer, 4 softmax warps, P V issuer
 constexpr int kStagesA = 2;
 constexpr uint32_t kIdescQK = idesc_bf16(BT, KT, false, false);
 struct SmemA {
   alignas(1024) unsigned char q[kTileBytes];
   alignas(1024) unsigned char k[kStagesA][kKvTileBytes];
   alignas(1024) unsigned char v[kStagesA][kKvTileBytes];
-  float xm[2][BT], xl[2][BT];              // row maxima / row sums of the two softmax warpgroups, exchanged
+  float xch[BT];
   uint64_t q_full, k_full[kStagesA], k_empty[kStagesA], v_full[kStagesA], v_empty[kStagesA];
   uint64_t s_full[2], p_full[2], pv_done[2];
   uint32_t tmem_base;
@@ -318,7 +318,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
     }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&sm.s_full[s], 1); mbar_init(&sm.pv_done[s], 1); mbar_init(&sm.p_full[s], 256);
+      mbar_init(&sm.s_full[s], 1); mbar_init(&sm.pv_done[s], 1); mbar_init(&sm.p_full[s], 128);
     }
     fence_barrier_init();
   }
@@ -367,7 +367,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         mma_commit(&sm.k_empty[st]);
       }
     }
-  } else if (warp == 10) {
+  } else if (warp == 6) {
     // ---- P V issuer: O += P V_j, 16 keys per step ----
     if (elect_one()) {
       for (int j = 0; j < nt; ++j) {
@@ -384,15 +384,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       }
     }
   } else {
-    // ---- softmax: thread (g, row) owns key columns [32g, 32g+32) of every tile of its query row ----
-    // The two threads of a row keep the same running maximum, so their halves of P feed ONE P V
-    // product. After the first tile P is formed speculatively with the maximum in use and only the
-    // tile sum is checked; a barrier that ORs "my half overflowed" over the 256 softmax threads is
-    // the only exchange a tile needs. When it says yes (rare), the halves' true maxima are exchanged
-    // through shared memory, the rows that grew are rescaled and P is formed again.
-    // A thread whose wait timed out (ok = false) keeps walking the loop and meeting the barriers, so
-    // that nobody waits at one for ever; it touches no data.
-    const int g = (warp - 2) >> 2;
+    // ---- softmax: one thread per query row, 64 logits per tile ----
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
     const int qpos = row0 + row;
@@ -402,34 +394,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     bool ok = true;
     for (int j = 0; j < nt; ++j) {
       const int sb = j & 1;
-      const int key0 = j * KT + 32 * g;                // first key of this thread's columns
-      if (ok && !mbar_wait(&sm.s_full[sb], (j >> 1) & 1)) { tf.raise(17); ok = false; }
-      ok = __all_sync(0xffffffffu, ok);                // the TMEM accesses below are warp-collective
+      const uint32_t colS = sb * KT;
+      if (!mbar_wait(&sm.s_full[sb], (j >> 1) & 1)) { tf.raise(17); ok = false; break; }
       tc_fence_after();
-      float s[32];
-      if (ok) {
-        uint32_t sr[32];
-        tmem_ld32(tmem + lane_base + sb * KT + 32 * g, sr);
-        tmem_wait_ld();
-        tmem_pin32(sr);
+      // the raw logits of this row (rs > 0, so the maximum can be taken before scaling)
+      uint32_t sa[32], sb2[32];
+      tmem_ld32(tmem + lane_base + colS, sa);
+      tmem_ld32(tmem + lane_base + colS + 32, sb2);
+      tmem_wait_ld();
+      tmem_pin32(sa);
+      tmem_pin32(sb2);
+      float s[64];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) s[c] = __uint_as_float(sr[c]);
-        if (key0 + 31 > row0) {                        // columns that cross the diagonal: causal mask
+      for (int c = 0; c < 32; ++c) { s[c] = __uint_as_float(sa[c]); s[32 + c] = __uint_as_float(sb2[c]); }
+      if (j * KT + KT - 1 > row0) {                    // a tile that crosses the diagonal: causal mask
 #pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (key0 + c > qpos) s[c] = -INFINITY;
-        }
-      } else {
-#pragma unroll
-        for (int c = 0; c < 32; ++c) s[c] = -INFINITY;
+        for (int c = 0; c < 64; ++c)
+          if (j * KT + c > qpos) s[c] = -INFINITY;
       }
-      uint32_t pk[16];
+      // P = 2^(S rs - m) as bf16 pairs (they will overwrite the first 32 columns of this S buffer) and their sum
+      uint32_t pk[32];
       float tile_sum = 0.f;
-      auto exp_pass = [&]() {                          // P = 2^(S rs - m) as bf16 pairs, and their sum
+      auto exp_pass = [&]() {
         const float neg_m = -m_used;
         float l4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
+        for (int c = 0; c < 32; ++c) {
           const float p0 = exp2f(fmaf(s[2 * c], rs, neg_m));
           const float p1 = exp2f(fmaf(s[2 * c + 1], rs, neg_m));
           l4[c & 3] += p0 + p1;
@@ -438,72 +428,67 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         }
         tile_sum = (l4[0] + l4[1]) + (l4[2] + l4[3]);
       };
-      bool redo = true;                                // the first tile has no maximum yet
+      // After the first tile the maximum in use is almost always good enough (a stale maximum only
+      // makes P, the row sum and O larger by the same factor), so P is formed SPECULATIVELY with it and
+      // the pass over the logits that takes their maximum is skipped: if the tile's probabilities add
+      // up to no more than kSpeculationLimit, none of them exceeds it and the tile stands. Otherwise
+      // (some row of the warp says so, or an overflow made the sum infinite) the maximum is taken
+      // properly, O is rescaled where needed and P is formed again.
+      bool settled = false;
       if (j > 0) {
         exp_pass();
-        redo = bar_or(1, 256, ok && !(tile_sum <= kSpeculationLimit));   // uniform over the 256 threads
+        settled = !__any_sync(0xffffffffu, !(tile_sum <= kSpeculationLimit));
       }
-      if (redo) {
-        float mx4[4] = {s[0], s[1], s[2], s[3]};
+      if (!settled) {
+        float mx4[4] = {s[0], s[1], s[2], s[3]};       // four chains of three-input maxima over s[4..63]
 #pragma unroll
-        for (int c = 4; c + 8 <= 32; c += 8) {         // s[4..27]
+        for (int c = 4; c + 8 <= 64; c += 8) {         // s[4..59]
 #pragma unroll
           for (int e = 0; e < 4; ++e) mx4[e] = max3(mx4[e], s[c + 2 * e], s[c + 2 * e + 1]);
         }
-        mx4[0] = max3(mx4[0], s[28], s[29]);
-        mx4[1] = max3(mx4[1], s[30], s[31]);
-        const float mx = fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]) * rs;   // -inf if all 32 columns are masked
-        sm.xm[g][row] = mx;
-        bar_sync(2, 256);
-        const float m_new = fmaxf(m_used, fmaxf(mx, sm.xm[1 - g][row]));     // the same in both threads of the row
+        mx4[0] = max3(mx4[0], s[60], s[61]);
+        mx4[1] = max3(mx4[1], s[62], s[63]);
+        const float mx = fmaxf(max3(mx4[0], mx4[1], mx4[2]), mx4[3]) * rs;   // -inf if the whole tile is masked for this row
+        const float m_new = fmaxf(m_used, mx);
         if (j == 0) {
           m_used = m_new;                              // finite: key 0 is never masked
         } else {
-          const bool need = ok && m_new > m_used + kRescaleThreshold;
-          if (__any_sync(0xffffffffu, need)) {         // the partner warp decides the same
+          const bool need = m_new > m_used + kRescaleThreshold;
+          if (__any_sync(0xffffffffu, need)) {
             const float alpha = need ? exp2f(m_used - m_new) : 1.0f;
             if (need) m_used = m_new;
             l *= alpha;
-            if (ok && !mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; }   // P V of tile j-1 landed
-            ok = __all_sync(0xffffffffu, ok);
+            if (!mbar_wait(&sm.pv_done[(j - 1) & 1], ((j - 1) >> 1) & 1)) { tf.raise(18); ok = false; break; }   // P V of tile j-1 landed
             tc_fence_after();
-            if (ok) {
 #pragma unroll 1
-              for (int c0 = 64 * g; c0 < 64 * g + 64; c0 += 32) {   // this warpgroup's half of the output columns
-                uint32_t r[32];
-                tmem_ld32(tmem + lane_base + kColO + c0, r);
-                tmem_wait_ld();
-                tmem_pin32(r);
+            for (int c0 = 0; c0 < D; c0 += 32) {
+              uint32_t r[32];
+              tmem_ld32(tmem + lane_base + kColO + c0, r);
+              tmem_wait_ld();
+              tmem_pin32(r);
 #pragma unroll
-                for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
-                tmem_st32(tmem + lane_base + kColO + c0, r);
-              }
-              tmem_wait_st();
+              for (int c = 0; c < 32; ++c) r[c] = __float_as_uint(__uint_as_float(r[c]) * alpha);
+              tmem_st32(tmem + lane_base + kColO + c0, r);
             }
+            tmem_wait_st();
           }
         }
         exp_pass();
       }
+      tmem_st32(tmem + lane_base + colS, pk);
       l += tile_sum;
-      if (ok) {
-        tmem_st16(tmem + lane_base + sb * KT + 16 * g, pk);
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(&sm.p_full[sb]);
-      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&sm.p_full[sb]);
     }
-    // ---- epilogue: the row sum is the two halves' sums; O / l -> bf16, row log2-sum-exp ----
+    // ---- epilogue: O / l -> bf16, row log2-sum-exp ----
     if (ok && !mbar_wait(&sm.pv_done[(nt - 1) & 1], ((nt - 1) >> 1) & 1)) { tf.raise(19); ok = false; }
-    ok = __all_sync(0xffffffffu, ok);
     tc_fence_after();
-    sm.xl[g][row] = l;
-    bar_sync(2, 256);
-    const float L = sm.xl[0][row] + sm.xl[1][row];
     if (ok) {
-      const float inv = 1.0f / L;
+      const float inv = 1.0f / l;
       __nv_bfloat16* orow = out + ((size_t)(tok0 + qpos) * Hq + h) * D;
 #pragma unroll 1
-      for (int c0 = 64 * g; c0 < 64 * g + 64; c0 += 32) {   // warpgroup g writes output columns [64g, 64g+64)
+      for (int c0 = 0; c0 < D; c0 += 32) {
         uint32_t r0[32];
         tmem_ld32(tmem + lane_base + kColO + c0, r0);
         tmem_wait_ld();
@@ -523,7 +508,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
           }
         }
       }
-      if (g == 0 && qpos < N) lse[(size_t)h * stride + lse_offset(tok0, b) + qpos] = m_used + log2f(L);
+      if (qpos < N) lse[(size_t)h * stride + lse_offset(tok0, b) + qpos] = m_used + log2f(l);
     }
   }
   tc_fence_before();
