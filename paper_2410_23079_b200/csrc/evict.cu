@@ -1,4 +1,4 @@
-// BUZZ eviction: segmented select-and-compact, one CTA at a time per (layer, sequence, KV head) instance.
+// BUZZ eviction: segmented select-and-compact, one CTA per (layer, sequence, KV head) instance.
 //
 // Algorithm 1 (sampling line + final concatenation) and Algorithm 2 of the paper:
 //   old region  [sink, sink + n_old)          keep offsets 0, s_hat, 2 s_hat, ...   (interval sampling)
@@ -34,9 +34,13 @@ __device__ inline Cand better(Cand a, Cand b) {
   return a;
 }
 
-// One instance, by the whole CTA. src: [budget] source slot of every destination slot (shared memory).
 template <int ROW_BYTES>
-__device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_t inst, int32_t* src) {
+__global__ void __launch_bounds__(kThreads)
+evict_kernel(BuzzState st, BuzzPolicy pol, int layer_begin, int max_batch, int kv_heads, int batch) {
+  extern __shared__ int32_t src[];   // [budget] source slot of every destination slot
+  const int head = blockIdx.x, seq = blockIdx.y, layer = layer_begin + blockIdx.z;
+  if (seq >= batch) return;
+  const size_t inst = ((size_t)layer * max_batch + seq) * kv_heads + head;
   const int n = st.n[inst];
   const int n_old = st.n_old[inst];
   if (n < pol.budget) return;                       // threshold buffering: evict only when full
@@ -141,23 +145,6 @@ __device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_
     st.n_old[inst] = kept_mid;
     if (n2 >= pol.budget) buzz_set_status(st.status, BUZZ_ERR_NO_PROGRESS, (int)inst, n2);
   }
-  __syncthreads();                                  // src[] is free for the CTA's next instance
-}
-
-// The CTAs walk the (layer, sequence, head) instances with a grid-sized stride. Most calls find
-// nothing due (the trigger is n >= budget), and then a launch costs a few counter reads per CTA
-// instead of one CTA per instance.
-template <int ROW_BYTES>
-__global__ void __launch_bounds__(kThreads)
-evict_kernel(BuzzState st, BuzzPolicy pol, int layer_begin, int layer_count, int max_batch, int kv_heads, int batch) {
-  extern __shared__ int32_t src[];
-  const int per_layer = batch * kv_heads;
-  const int total = layer_count * per_layer;
-  for (int idx = blockIdx.x; idx < total; idx += gridDim.x) {
-    const int l = idx / per_layer, rem = idx - l * per_layer;
-    const int seq = rem / kv_heads, head = rem - seq * kv_heads;
-    evict_instance<ROW_BYTES>(st, pol, ((size_t)(layer_begin + l) * max_batch + seq) * kv_heads + head, src);
-  }
 }
 
 }  // namespace
@@ -166,30 +153,21 @@ cudaError_t buzz_launch_evict(buzz_ctx* c, int layer_begin, int layer_count, cud
   int batch = 0;
   for (int l = layer_begin; l < layer_begin + layer_count; ++l) batch = max(batch, c->batch[l]);
   if (batch == 0) return cudaSuccess;
-  const long total = (long)c->sh.kv_heads * batch * layer_count;
-  unsigned grid = 0;                                 // one resident wave of CTAs, or fewer if there is less to do
+  dim3 grid(c->sh.kv_heads, batch, layer_count);
   (void)cudaGetLastError();   // drop a stale non-sticky error left by an earlier runtime call of the process
   const size_t smem = (size_t)c->pol.budget * sizeof(int32_t);
   const int row_bytes = c->sh.head_dim * (int)c->esize;
 #define BUZZ_EVICT_CASE(RB)                                                                        \
   case RB: {                                                                                       \
     static bool attr_done = false;                                                                 \
-    static int sms = 0;                                                                            \
     if (!attr_done) {                                                                              \
       cudaError_t e = cudaFuncSetAttribute(evict_kernel<RB>,                                       \
                                            cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); \
       if (e != cudaSuccess) return e;                                                              \
-      int dev = 0;                                                                                 \
-      if (cudaGetDevice(&dev) != cudaSuccess ||                                                    \
-          cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return cudaErrorUnknown; \
       attr_done = true;                                                                            \
     }                                                                                              \
-    int per_sm = 0;                                                                                \
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, evict_kernel<RB>, kThreads, smem) != cudaSuccess || per_sm < 1) \
-      return cudaErrorInvalidValue;                                                                \
-    grid = (unsigned)(total < (long)per_sm * sms ? total : (long)per_sm * sms);                    \
-    evict_kernel<RB><<<grid, kThreads, smem, stream>>>(c->st, c->pol, layer_begin, layer_count,      \
-                                                       c->sh.max_batch, c->sh.kv_heads, batch);    \
+    evict_kernel<RB><<<grid, kThreads, smem, stream>>>(c->st, c->pol, layer_begin, c->sh.max_batch, \
+                                                       c->sh.kv_heads, batch);                     \
     break;                                                                                         \
   }
   switch (row_bytes) {
