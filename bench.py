@@ -322,9 +322,9 @@ def run_ours(args):
                h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h)
     assert bz.status() == 0
 
-    # ---- eviction leg: keep decoding until the first decode-time eviction, time that call ----
-    evict = None
-    if not args.no_evict_leg:
+    # ---- eviction leg: keep decoding until the first, then the second, decode-time eviction; time those calls ----
+    def timed_eviction():
+        nonlocal t
         guard = 0
         while max(n for n, _ in counts) + 1 < w.budget and guard < 5000:
             step(t); bz.evict(-1); advance_counts(); t += 1; guard += 1
@@ -344,9 +344,14 @@ def run_ours(args):
             if fired:
                 moved += 4 * (n - w.sink - w.window) + 2 * (n2 - w.sink) * per_slot   # scan + rows read and written
         ev_bytes = moved * w.kv_heads * w.layers
-        evict = dict(ms=ev_ms, sequences_evicting=sum(1 for n, _ in before if n >= w.budget),
-                     gbs=ev_bytes / (ev_ms * 1e-3) / 1e9, frac_of_hbm_peak=ev_bytes / (ev_ms * 1e-3) / 1e9 / peaks["hbm"],
-                     bytes=ev_bytes, at_step=t)
+        return dict(ms=ev_ms, sequences_evicting=sum(1 for n, _ in before if n >= w.budget),
+                    gbs=ev_bytes / (ev_ms * 1e-3) / 1e9, frac_of_hbm_peak=ev_bytes / (ev_ms * 1e-3) / 1e9 / peaks["hbm"],
+                    bytes=ev_bytes, at_step=t)
+
+    evict = None
+    if not args.no_evict_leg:
+        evict = timed_eviction()
+        evict["second"] = timed_eviction()             # old and new tokens both present this time
         assert bz.status() == 0
 
     line = dict(metric="decode tokens/s (attention + BUZZ eviction)", value=whole_job_rate(w.batch * K, world, ms),
