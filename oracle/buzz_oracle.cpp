@@ -19,6 +19,9 @@
 //                                (Section 3.3, "BeeHive" and the sentence introducing Alg. 1/2).
 //   * short sequences          : Remark 1 (nothing is evicted while n <= k + w).
 //   * over-long prompts        : Remark 2 (sample repeatedly until the cache fits T + k + w).
+//   * log-n scaled attention   : Section 3.5 (logits scaled by log_512(n)/sqrt(d), n = tokens seen so
+//                                far: row index + 1 at prefill, total length incl. the new token at
+//                                decode -- not the number of retained slots).
 //
 // Readings taken where the paper is silent or inconsistent (each also listed in the design notes):
 //   T is the capacity of the middle region, budget = T + k + w (Remark 2, Fig. 3 caption);

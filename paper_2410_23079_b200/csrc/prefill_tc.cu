@@ -389,7 +389,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     const int row = quarter * 32 + lane;
     const int qpos = row0 + row;
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    const float rs = scale_log2 * (logn ? __logf((float)(qpos + 1)) * kInvLn512 : 1.0f);
+    // Row scale. With log-n scaling the first row of a sequence has log_512(1) = 0: its only unmasked
+    // logit is scaled to 0 and its probability is 1. The scale is kept a hair above zero there so that
+    // a masked logit (-inf) times the scale stays -inf instead of becoming NaN; a finite logit times
+    // 1e-30 is 0 to far below fp32 resolution, so row 0 still gets exactly P = 1.
+    const float rs = logn ? fmaxf(scale_log2 * __logf((float)(qpos + 1)) * kInvLn512, 1e-30f) : scale_log2;
     float m_used = -INFINITY, l = 0.f;
     bool ok = true;
     for (int j = 0; j < nt; ++j) {
@@ -397,7 +401,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
       const uint32_t colS = sb * KT;
       if (!mbar_wait(&sm.s_full[sb], (j >> 1) & 1)) { tf.raise(17); ok = false; break; }
       tc_fence_after();
-      // the raw logits of this row (rs > 0, so the maximum can be taken before scaling)
+      // the raw logits of this row (rs > 0 always, see above, so the maximum can be taken before scaling)
       uint32_t sa[32], sb2[32];
       tmem_ld32(tmem + lane_base + colS, sa);
       tmem_ld32(tmem + lane_base + colS + 32, sb2);

@@ -41,12 +41,37 @@ def test_handworked_case():
     assert h.counts()[:2] == (len(b["expect_pos"]), b["expect_n_old"])
 
 
+def _evict_full_cache(h, sink, window, budget, n_old, rng):
+    """Plants a full cache (n = budget, of which n_old slots are old, random scores) and runs ONE
+    eviction of the oracle; returns the retained original slot indices."""
+    pos = np.arange(budget, dtype=np.int32)
+    K = pos[:, None].astype(np.float64)
+    h.set_state(n_old, budget, pos, rng.random(budget), K, -K)
+    assert h.evict() == 1
+    return h.state(with_kv=False)[0].tolist()
+
+
 def test_paper_printed_values():
+    """The two numbers the paper prints for stride 5, observed on the oracle's behaviour: s_hat = 3
+    (which old slots survive one eviction) and the optimum T/w = 4.33 (the ratio of the middle
+    region's capacity to the steady-state number of old tokens, which the theorem equates with w)."""
     with open(os.path.join(GOLD, "paper_values.json")) as f:
         gold = json.load(f)
     s = gold["t_over_w_s5"]["s"]
-    assert (s + 1) // 2 == gold["s_hat_formula"]["s_hat"]
-    assert abs((s * s + 1) / (s + 1) - gold["t_over_w_s5"]["value"]) <= gold["t_over_w_s5"]["abs_tol"]
+    assert s == gold["s_hat_formula"]["s"]
+    s_hat = gold["s_hat_formula"]["s_hat"]
+    rng = np.random.default_rng(0)
+    sink, window, T = 2, 7, 26000
+    budget = sink + window + T
+    h = OracleHead(1, 1, sink, window, s, 1, budget)
+    kept = _evict_full_cache(h, sink, window, budget, 100, rng)
+    old_kept = [p - sink for p in kept if sink <= p < sink + 100]
+    assert old_kept == list(range(0, 100, s_hat))                  # every s_hat-th old slot, from offset 0
+    a = h.counts()[1]
+    for _ in range(60):                                            # iterate eviction on a full cache to steady state
+        _evict_full_cache(h, sink, window, budget, a, rng)
+        a = h.counts()[1]
+    assert abs(T / a - gold["t_over_w_s5"]["value"]) <= gold["t_over_w_s5"]["abs_tol"]
 
 
 def _run_schedule(sink, window, s, hitters, budget, evictions, seed=0):
@@ -85,6 +110,31 @@ def test_count_recursion_and_steady_state(s):
     assert seq == _run_schedule(sink, window, s, 1, budget, 60, seed=s + 100)   # score-independent
     fixed = T * (s + 1) / (s * s + 1) if s % 2 else T / (s - 1)
     assert abs(seq[-1] - fixed) <= 3.0
+
+
+@pytest.mark.parametrize("s,hitters", [(3, 1), (4, 1), (5, 1), (5, 2), (8, 1), (16, 2), (31, 3)])
+def test_count_recursion_over_1000_evictions(s, hitters):
+    """1000 consecutive evictions of a refilled cache: after every one, n_old equals the integer
+    recursion a' = ceil(a/s_hat) + kept((T - a), s, h) with kept(m) = (ceil(m/s) - 1) h + min(h, last
+    segment), whatever the scores; for one hitter per segment the sequence settles within the proof's
+    slack of the theorem's fixed point (Appendix C.1)."""
+    sink, window, T = 3, 20, 997
+    budget = sink + window + T
+    s_hat = (s + 1) // 2
+    rng = np.random.default_rng(s * 7 + hitters)
+    h = OracleHead(1, 1, sink, window, s, hitters, budget)
+    a = 0
+    for it in range(1000):
+        _evict_full_cache(h, sink, window, budget, a, rng)
+        m = T - a
+        nseg = math.ceil(m / s)
+        kept_new = 0 if nseg == 0 else (nseg - 1) * hitters + min(hitters, m - (nseg - 1) * s)
+        a = math.ceil(a / s_hat) + kept_new
+        n, n_old, _ = h.counts()
+        assert n_old == a and n == sink + a + window < budget, f"eviction {it}"
+    if hitters == 1:
+        fixed = T * (s + 1) / (s * s + 1) if s % 2 else T / (s - 1)
+        assert abs(a - fixed) <= 3.0
 
 
 def test_first_eviction_shrinks_middle_by_s_minus_1_over_s():
