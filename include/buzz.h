@@ -67,15 +67,20 @@ enum {
  *             counters n / n_old / total_len [L][max_batch][Hkv], and the status words.
  *   scratch : per-row softmax statistics and per-key column sums of one prefill, plus staging
  *             buffers (one set per layer) for the host-buffer decode entries. Contents are not carried between calls.
- * Returns BUZZ_ERR_INVALID for a shape or budget the library does not support. */
+ * Returns BUZZ_ERR_INVALID for a shape or budget the library does not support: any of layers,
+ * max_batch, q_heads, kv_heads, max_prompt_tokens < 1; kv_heads not dividing q_heads; a group size
+ * q_heads / kv_heads other than 1, 2, 4 or 8; head_dim other than 64 or 128; an unknown dtype;
+ * budget < 1 or budget > 32768; a null pointer. */
 int buzz_workspace_bytes(const buzz_shape* shape, int budget, size_t* state_bytes, size_t* scratch_bytes);
 
 /* Creates a cache policy object (Table 1: k = sink, w = window, s = segment; budget = T + k + w,
  * Remark 2). `hitters` is the number of winners kept per segment. Both allocations must be at
  * least as large as buzz_workspace_bytes reports and 256-byte aligned; `state_dev` is zeroed here
- * (one synchronous memset on the default stream). Rejects: sink < 0, window < 1, segment < 2,
- * hitters < 1, hitters >= segment, budget < sink + window + segment, kv_heads not dividing
- * q_heads, head_dim not in {64, 128}, undersized or misaligned buffers. */
+ * (one synchronous memset on the default stream). The device that is current at this call is the
+ * one the object's kernels are sized for.
+ * Rejects (BUZZ_ERR_INVALID, nothing allocated): everything buzz_workspace_bytes rejects; sink < 0;
+ * window < 1; segment < 2 or segment > 1024; hitters < 1 or hitters >= segment;
+ * budget < sink + window + segment; null, undersized or misaligned buffers. */
 int buzz_create(buzz_t* out, int sink, int window, int segment, int hitters, int budget,
                 const buzz_shape* shape, void* state_dev, size_t state_bytes,
                 void* scratch_dev, size_t scratch_bytes);
@@ -85,14 +90,17 @@ void buzz_destroy(buzz_t ctx);
 
 /* Prefill of one layer (Eqs. 1 and 3; Remark 2).
  *   q  [total_tokens][Hq][d], k, v [total_tokens][Hkv][d], out [total_tokens][Hq][d], all packed
- *   over `batch` sequences by cu_seqlens_dev [batch+1] (int32, device; cu[0] = 0).
+ *   over `batch` sequences by cu_seqlens_dev [batch+1] (int32, device; cu[0] = 0, non-decreasing,
+ *   cu[batch] = total_tokens -- the library never reads the array on the host and does not verify it).
  * Computes causal attention out = Softmax(q k^T / sqrt(d)) v per sequence and head, the initial
  * score of every key = the sum of the probabilities it received (column sums, summed over the
  * query heads of its group, in a fixed order), then, while a sequence holds >= budget tokens,
  * eviction rounds (first round: segment-wise top-`hitters` over everything between sink and
  * window; later rounds: every s_hat-th survivor), and writes the survivors' K, V, score and
  * position into the layer's cache. Resets that layer's sequences 0..batch-1.
- * `max_seqlen` is an upper bound on any sequence's length (host value, used for grid sizing). */
+ * `max_seqlen` is an upper bound on any sequence's length (host value, used for grid sizing).
+ * Rejects: layer outside [0, layers); batch < 1 or > max_batch; total_tokens < 1 or
+ * > max_prompt_tokens; max_seqlen < 1 or > total_tokens; null or misaligned pointers. */
 int buzz_prefill(buzz_t ctx, int layer, const void* q, const void* k, const void* v,
                  const int32_t* cu_seqlens_dev, int batch, int total_tokens, int max_seqlen,
                  void* out, void* stream);
@@ -107,15 +115,23 @@ int buzz_prefill(buzz_t ctx, int layer, const void* q, const void* k, const void
  * holds that array until the process exits.
  *   - Limit: (q_heads + kv_heads) * total_tokens <= BUZZ_STATIC_SCRATCH_FLOATS (1,048,576 floats);
  *     larger calls return BUZZ_ERR_TOO_LARGE and launch nothing. total_tokens need not respect
- *     max_prompt_tokens.
+ *     max_prompt_tokens. cu_seqlens_dev[batch] must equal total_tokens as for buzz_prefill: an
+ *     array that runs past it would make the kernels write beyond the built-in array.
+ *   - Kernels: this entry always runs the library's CUDA-core (fp32-pipe) prefill kernels, also for
+ *     bf16 with head_dim 128 where buzz_prefill uses the tensor-core kernels; it is meant for
+ *     modest prompts. Outputs agree with buzz_prefill's within the library's tolerances and the
+ *     scores to rel 1e-3, not bit for bit, so where two candidates of a segment are tied to that
+ *     precision the two entries may retain different tokens.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress) with
- *     that device current; make that first call outside any stream capture.
- *   - The call allocates and frees nothing. All calls on a device share the array, which keeps
- *     the previous call's contents (each call overwrites every entry before reading it, so no
- *     clearing is needed); calls whose kernels overlap on the GPU race on it, so order them on
- *     one stream or with events.
+ *     that device current; make that first call outside any stream capture. If the process has not
+ *     yet run any of the library's kernels on that device, that first call is also when the driver
+ *     loads the library's device code and places the array, which is a driver-side allocation; from
+ *     the second call on a device on, nothing is allocated or freed.
+ *   - All calls on a device share the array, which keeps the previous call's contents (each call
+ *     overwrites every entry before reading it, so no clearing is needed); calls whose kernels
+ *     overlap on the GPU race on it, so order them on one stream or with events.
  *   - buzz_export_prefill_scores does not see this call's scores (they are in the built-in array).
- * Arguments, results, cache update and error behaviour are otherwise those of buzz_prefill. */
+ * Arguments, cache update and error behaviour are otherwise those of buzz_prefill. */
 #define BUZZ_STATIC_SCRATCH_FLOATS (1u << 20)
 int buzz_prefill_static(buzz_t ctx, int layer, const void* q, const void* k, const void* v,
                         const int32_t* cu_seqlens_dev, int batch, int total_tokens, int max_seqlen,

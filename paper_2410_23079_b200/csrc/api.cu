@@ -134,6 +134,15 @@ int buzz_create(buzz_t* out, int sink, int window, int segment, int hitters, int
   c->stage_kv = L.stage_kv;
   c->batch = static_cast<int*>(calloc(shape->layers, sizeof(int)));
   c->decode_cluster = 0;
+  c->sm_count = 148;
+  {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      c->sm_count = sms;
+    else
+      (void)cudaGetLastError();
+  }
   c->launches = 0;
   c->last_kind = 0; c->last_layer = -1; c->last_stream = nullptr;
   if (!c->batch) { delete c; return BUZZ_ERR_INVALID; }

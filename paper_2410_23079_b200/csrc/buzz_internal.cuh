@@ -46,6 +46,7 @@ struct buzz_ctx {
   size_t stage_q, stage_kv;  // byte sizes of one q-shaped and one kv-shaped staging tensor
   int* batch;         // active sequences per layer (host array)
   int decode_cluster; // 0 = choose automatically
+  int sm_count;       // multiprocessors of the device that was current at buzz_create
   long long launches;
   // what the library launched last through this object (0 nothing, 1 a bf16 decode step, 2 anything else)
   int last_kind, last_layer;
@@ -63,6 +64,25 @@ __device__ inline void buzz_set_status(int32_t* status, int code, int inst, int 
     status[2] = detail;
   }
 }
+
+// The opt-in to more than 48 KB of dynamic shared memory is a per-DEVICE property of a kernel. One of
+// these per kernel (a function-local static) remembers, per device ordinal, the largest size already
+// applied, so that a process driving several GPUs sets it on each of them.
+constexpr int kBuzzMaxDevices = 64;
+struct BuzzSmemOptIn {
+  size_t applied[kBuzzMaxDevices] = {};
+  template <typename Kernel>
+  cudaError_t ensure(Kernel kernel, size_t bytes) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kBuzzMaxDevices) return cudaErrorInvalidDevice;
+    if (bytes <= applied[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess) applied[dev] = bytes;
+    return e;
+  }
+};
 
 // ---- launch wrappers (each returns a cudaError_t from the launch) ---------------------------
 // chain_pos: -1 for a single-layer call, else the index of this launch within one multi-layer call

@@ -293,12 +293,8 @@ cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, con
   const int chunk_cap = (c->pol.budget + cluster_size - 1) / cluster_size;
   const size_t smem = sizeof(Partial<G, D>) +
                       sizeof(float) * (kWarps * G + kMaxCluster * G + G + kWarps * G * D + (size_t)G * chunk_cap);
-  static size_t smem_set = 0;
-  if (smem > smem_set) {
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel<T, D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    smem_set = smem;
-  }
+  static BuzzSmemOptIn opt_in;
+  if (cudaError_t e = opt_in.ensure(decode_kernel<T, D, G>, smem); e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(cluster_size, c->sh.kv_heads, batch);
   cfg.blockDim = dim3(kThreads);
@@ -342,11 +338,11 @@ cudaError_t buzz_launch_decode(buzz_ctx* c, int layer, const void* q, const void
   int cs = c->decode_cluster;
   if (cs == 0) {
     // The whole grid should be one resident wave of long-lived CTAs: the smallest power-of-two
-    // split that gives every one of the 148 SMs at least one or two CTAs (measured best on C2 and
+    // split that gives every SM (148 on a B200) at least one or two CTAs (measured best on C2 and
     // C4 shapes), while every CTA still streams at least ~64 rows.
     const long inst = (long)c->batch[layer] * c->sh.kv_heads;
     cs = 1;
-    while (cs < kMaxCluster && inst * cs < 148L * 3 / 2 && (c->pol.budget / (cs * 2)) >= 64) cs *= 2;
+    while (cs < kMaxCluster && inst * cs < (long)c->sm_count * 3 / 2 && (c->pol.budget / (cs * 2)) >= 64) cs *= 2;
   }
   // the logits of a chunk must fit in shared memory
   while (cs < kMaxCluster && (size_t)c->group * ((c->pol.budget + cs - 1) / cs) * sizeof(float) > 96 * 1024) cs *= 2;

@@ -375,12 +375,8 @@ cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, con
                       sizeof(float) * (kWarps * kHeads + kHeads + kMaxCluster * G + 2 * G +
                                        kWarps * G * D + (size_t)G * chunk_cap);
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
-  static size_t smem_set = 0;
-  if (smem > smem_set) {
-    cudaError_t e = cudaFuncSetAttribute(decode_bf16_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    smem_set = smem;
-  }
+  static BuzzSmemOptIn opt_in;
+  if (cudaError_t e = opt_in.ensure(decode_bf16_kernel<D, G>, smem); e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(cluster_size, c->sh.kv_heads, batch);
   cfg.blockDim = dim3(kThreads);

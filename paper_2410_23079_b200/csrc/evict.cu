@@ -159,13 +159,8 @@ cudaError_t buzz_launch_evict(buzz_ctx* c, int layer_begin, int layer_count, cud
   const int row_bytes = c->sh.head_dim * (int)c->esize;
 #define BUZZ_EVICT_CASE(RB)                                                                        \
   case RB: {                                                                                       \
-    static bool attr_done = false;                                                                 \
-    if (!attr_done) {                                                                              \
-      cudaError_t e = cudaFuncSetAttribute(evict_kernel<RB>,                                       \
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); \
-      if (e != cudaSuccess) return e;                                                              \
-      attr_done = true;                                                                            \
-    }                                                                                              \
+    static BuzzSmemOptIn opt_in;                                                                   \
+    if (cudaError_t e = opt_in.ensure(evict_kernel<RB>, smem); e != cudaSuccess) return e;         \
     evict_kernel<RB><<<grid, kThreads, smem, stream>>>(c->st, c->pol, layer_begin, c->sh.max_batch, \
                                                        c->sh.kv_heads, batch);                     \
     break;                                                                                         \

@@ -8,6 +8,11 @@
 // sums, normally part of the scratch allocation given to buzz_create). Here they live in one
 // fixed array that the library image itself carries.
 //
+// Which kernels: always the CUDA-core (fp32-pipe) prefill kernels, whatever the dtype and head
+// dimension, because their two temporaries are plain [heads][total_tokens] arrays that fit the
+// built-in array exactly (the tensor-core kernels want padded, aligned row statistics). The results
+// agree with buzz_prefill's within the library's tolerances, scores to rel 1e-3, not bit for bit.
+//
 // Cost and limits: the array takes BUZZ_STATIC_SCRATCH_FLOATS * 4 bytes (4 MiB) on every GPU that
 // loads the library, until the process exits. A call needs (q_heads + kv_heads) * total_tokens
 // floats and is refused with BUZZ_ERR_TOO_LARGE if that exceeds the array. All calls on a device
@@ -69,6 +74,7 @@ extern "C" int buzz_prefill_static(buzz_t c, int layer, const void* q, const voi
   buzz_ctx view = *c;
   view.sh.max_prompt_tokens = total_tokens;
   view.lse = base;
+  view.lse_stride = total_tokens;   // unused by the CUDA-core kernels (their row stride is max_prompt_tokens)
   view.pscore = base + (size_t)c->sh.q_heads * total_tokens;
   view.launches = 0;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

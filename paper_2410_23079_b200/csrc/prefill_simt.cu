@@ -217,14 +217,9 @@ cudaError_t launch_simt(buzz_ctx* c, const void* q, const void* k, const void* v
   constexpr int LD = D + 4;
   const size_t smemA = sizeof(float) * (BM * LD + 2 * BN * LD + BM * (BN + 4));
   const size_t smemB = sizeof(float) * (BM * LD + BN * LD + BM + 16 * BN);
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(prefill_attn_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smemA);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(prefill_colsum_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smemB);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
+  static BuzzSmemOptIn opt_in_a, opt_in_b;
+  if (cudaError_t e = opt_in_a.ensure(prefill_attn_kernel<T, D>, smemA); e != cudaSuccess) return e;
+  if (cudaError_t e = opt_in_b.ensure(prefill_colsum_kernel<T, D>, smemB); e != cudaSuccess) return e;
   const int tiles = (max_seqlen + BM - 1) / BM;
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
   const int logn = (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0;

@@ -564,14 +564,9 @@ cudaError_t buzz_launch_prefill_tc(buzz_ctx* c, const void* q, const void* k, co
       !make_map(&mk64, k, total_tokens, c->sh.kv_heads, KT) || !make_map(&mv64, v, total_tokens, c->sh.kv_heads, KT))
     return cudaErrorInvalidValue;
   const size_t smemA = sizeof(SmemA) + 1024, smemB = sizeof(SmemB) + 1024;
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smemA);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smemB);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
+  static BuzzSmemOptIn opt_in_a, opt_in_b;
+  if (cudaError_t e = opt_in_a.ensure(attn_tc_kernel, smemA); e != cudaSuccess) return e;
+  if (cudaError_t e = opt_in_b.ensure(colsum_tc_kernel, smemB); e != cudaSuccess) return e;
   const int tiles = (max_seqlen + BT - 1) / BT;
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
   const int logn = (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0;

@@ -7,7 +7,12 @@ sampled (layer, sequence, KV head) instance:
     which then takes every arg-max decision on exactly the values the GPU holds; retained
     positions, counters, scores and K/V rows must then match bit for bit;
   * every decode step's output is compared within tolerance, the running scores to rel 1e-3, and
-    before each eviction the oracle's scores are replaced by the GPU's (lock-step again).
+    before each eviction the oracle's scores are replaced by the GPU's (lock-step again);
+  * where the oracle ran the whole prefill, a third, FREE-RUNNING oracle instance never sees the
+    GPU's scores: at every eviction its retained positions are compared with the GPU's, and every
+    difference must be a near-tie (the two candidates' scores, in the oracle's own fp64, within rel
+    1e-3 of each other, inside one segment); after a difference it is re-aligned with the lock-step
+    instance, because the trajectories legitimately part from there.
 """
 from __future__ import annotations
 
@@ -62,6 +67,27 @@ def compare_state(bz: Buzz, orc: OracleHead, layer, seq, head, what, exact_score
     return st
 
 
+def check_free_running(fr: OracleHead, before, gpu_pos, w, what, stats):
+    """`before` = (pos, score) of the free-running oracle just before its eviction, `gpu_pos` the
+    positions the GPU retained. Counts are score-independent, so the two retained sets have the same
+    size; positions only one side kept are paired in order and each pair must be a near-tie."""
+    pos_b, sc_b = before
+    score_of = dict(zip(pos_b.tolist(), sc_b.tolist()))
+    slot_of = {p: i for i, p in enumerate(pos_b.tolist())}
+    mine = fr.state(with_kv=False)[0].tolist()
+    only_f = sorted(set(mine) - set(gpu_pos))
+    only_g = sorted(set(gpu_pos) - set(mine))
+    assert len(only_f) == len(only_g), f"{what}: free-running oracle and GPU kept different counts"
+    for pf, pg in zip(only_f, only_g):
+        a, b = score_of[pf], score_of[pg]
+        assert abs(a - b) <= SCORE_RTOL * max(abs(a), abs(b)), \
+            f"{what}: GPU kept position {pg} (score {b}) where the oracle kept {pf} (score {a}): not a near-tie"
+        assert abs(slot_of[pf] - slot_of[pg]) < fr.segment, f"{what}: positions {pf}, {pg} are not in one segment"
+    stats["free_running_evictions"] += 1
+    stats["free_running_near_ties"] += len(only_f)
+    return len(only_f) == 0
+
+
 def check_prefill_sampled(w, Q, K, V, got, gpu_scores, rows, tail_keys, tol, logn, what, stats):
     """Full-size prefill check without the O(N^2) oracle prefill. Row i of causal attention is one
     decode step of the oracle over the prefix [0, i) (Eq. 3 for one query), so sampled output rows
@@ -104,8 +130,9 @@ def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None,
     lens = workloads.prompt_lengths(w)
     offs = np.concatenate([[0], np.cumsum(lens)])
     g, d = w.group, w.head_dim
-    stats = dict(evictions=0, prefill_rounds=0, max_out_err=0.0)
+    stats = dict(evictions=0, prefill_rounds=0, max_out_err=0.0, free_running_evictions=0, free_running_near_ties=0)
     lock = {}
+    frees = {}
     dec = {}
     for layer in layers:
         q, k, v, cu = workloads.prefill_inputs(w, layer, device)
@@ -133,6 +160,7 @@ def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None,
                 assert_close(got, O, what=f"prefill out L{layer} b{b} h{h}", **tol)
                 stats["max_out_err"] = max(stats["max_out_err"], float(np.abs(got - O).max()))
                 assert_scores_close(gs, full, f"prefill scores L{layer} b{b} h{h}")
+                frees[(layer, b, h)] = free
             else:
                 check_prefill_sampled(w, Q, K, V, got, gs, sampled_rows, tail_keys, tol, logn,
                                       f"L{layer} b{b} h{h}", stats)
@@ -144,8 +172,19 @@ def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None,
             ls.set_state(0, N, np.arange(N), gs.astype(np.float64), K, V)
             while ls.counts()[0] >= w.budget:
                 assert ls.evict() == 1
-            compare_state(bz, ls, layer, b, h, f"after prefill L{layer} b{b} h{h}", exact_scores=True)
+            st0 = compare_state(bz, ls, layer, b, h, f"after prefill L{layer} b{b} h{h}", exact_scores=True)
             lock[(layer, b, h)] = ls
+            fr = frees.get((layer, b, h))
+            if fr is not None and fr.counts()[0] != e - a:      # the free-running oracle sampled at prefill too
+                if rounds == 1:                                 # one round: every difference must be a near-tie
+                    same = check_free_running(fr, (np.arange(N), full), st0["pos"].tolist(), w,
+                                              f"prefill sampling L{layer} b{b} h{h}", stats)
+                else:                                           # later rounds thin by index: one near-tie shifts the rest
+                    same = fr.state(with_kv=False)[0].tolist() == st0["pos"].tolist()
+                    stats["free_running_evictions"] += 1
+                    stats["free_running_near_ties"] += 0 if same else 1
+                if not same:
+                    fr.set_state(ls.counts()[1], ls.counts()[2], *ls.state())
     for t in range(S):
         outs = {layer: torch.empty_like(dec[layer][0][t]) for layer in layers}
         if layers_call:                          # the whole stack in one multi-layer call
@@ -169,6 +208,10 @@ def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None,
                 if will_evict:
                     ls.set_scores(st["score"].numpy().astype(np.float64))
             pre[key] = will_evict
+            fr = frees.get(key)
+            if fr is not None:
+                ref_f = fr.decode(_np64(qd[t, b, h * g:(h + 1) * g]), _np64(kd[t, b, h]), _np64(vd[t, b, h]))
+                assert_close(got, ref_f, what=f"decode out step {t} {key} (free-running oracle)", **tol)
         for layer in layers:
             bz.evict(layer)
         assert bz.status() == 0, f"device status after step {t}"
@@ -177,7 +220,13 @@ def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None,
             assert r == (1 if pre[key] else 0)
             if pre[key]:
                 stats["evictions"] += 1
-                compare_state(bz, ls, *key, f"after eviction step {t} {key}", exact_scores=True)
+                st = compare_state(bz, ls, *key, f"after eviction step {t} {key}", exact_scores=True)
+                fr = frees.get(key)
+                if fr is not None:
+                    before = fr.state(with_kv=False)
+                    assert fr.evict() == 1
+                    if not check_free_running(fr, before, st["pos"].tolist(), w, f"eviction step {t} {key}", stats):
+                        fr.set_state(ls.counts()[1], ls.counts()[2], *ls.state())
     if own:
         bz.close()
     return stats

@@ -45,3 +45,10 @@ def test_c2_full_shape_extended_decode_eviction(cuda_device):
     w = workloads.scaled(workloads.get("C2"), layers=1, decode_steps=885)
     stats = run_lockstep(w, [(0, 0, 0), (0, 7, 31)], sampled_rows=_rows(4096), tail_keys=32, check_every=64)
     assert stats["evictions"] == 2
+
+
+def test_c2_full_shape_one_layer_logn(cuda_device):
+    """One full-shape C2 layer with log_512(n) logit scaling (Section 3.5): sampled rows (the first
+    token of a sequence, whose scale is zero, among them), tail column sums, lock-step decode."""
+    w = workloads.scaled(workloads.get("C2"), layers=1, decode_steps=3)
+    run_lockstep(w, [(0, 0, 0), (0, 5, 19)], sampled_rows=_rows(4096), tail_keys=48, logn=True)

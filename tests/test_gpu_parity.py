@@ -60,6 +60,24 @@ def test_logn_scaling(cuda_device):
     run_lockstep(w, [(0, 0, 0)], logn=True)
 
 
+@pytest.mark.parametrize("name,over,samples", [
+    ("C2", dict(layers=2, batch=2, q_heads=4, kv_heads=4, prompt_min=700, prompt_max=700, decode_steps=150,
+                window=64, budget=180), [(0, 0, 0), (1, 1, 3)]),
+    ("C4", dict(layers=1, batch=2, q_heads=8, kv_heads=2, prompt_min=900, prompt_max=900, decode_steps=130,
+                window=64, budget=300), [(0, 1, 0), (0, 0, 1)]),
+    ("C5", dict(layers=1, batch=3, q_heads=2, kv_heads=2, prompt_min=130, prompt_max=600, decode_steps=60,
+                window=48, budget=200), [(0, 0, 0), (0, 1, 1), (0, 2, 0)]),
+])
+def test_logn_scaling_on_the_tensor_core_path(cuda_device, name, over, samples):
+    """log_512(n) scaling on bf16, d = 128: the TMA/tcgen05 prefill kernels (prompts of several key
+    tiles with a ragged tail, MHA and GQA) and the tensor-core decode kernel, through prefill-time
+    sampling rounds and decode-time evictions (where tokens seen and retained slots differ). Every
+    output row is compared, so the first token of each sequence (scale 0) is covered."""
+    w = workloads.scaled(workloads.get(name), **over)
+    stats = run_lockstep(w, samples, check_every=7, logn=True)
+    assert stats["evictions"] >= 2 and np.isfinite(stats["max_out_err"])
+
+
 @pytest.mark.parametrize("N", [1, 3, 40, 68, 69, 159, 160, 161, 700])
 def test_prompt_length_edges(cuda_device, N):
     """Prompts shorter than sink+window (Remark 1), just below / at / above the budget, and far
