@@ -216,6 +216,15 @@ int buzz_export_prefill_scores(buzz_t ctx, int kv_head, int total_tokens, float*
  * (BUZZ_OK if none) and clears it. */
 int buzz_status(buzz_t ctx, void* stream);
 
+/* Self-test of the failure-detection path (not part of the method). Every wait inside the library's
+ * kernels is bounded: after a fixed number of polls it gives up, records BUZZ_ERR_TIMEOUT in the
+ * device status word and the kernel runs to its end. This call makes that happen on purpose and
+ * harmlessly: one small CTA waits, through the same bounded wait, on a barrier at which nobody ever
+ * arrives, with a limit of `polls` polls (1..65536; each poll may itself block for a few
+ * microseconds). The kernel ends by itself; afterwards buzz_status() returns BUZZ_ERR_TIMEOUT once
+ * and the object stays fully usable. No cache contents are touched. */
+int buzz_selftest_wait_expiry(buzz_t ctx, int polls, void* stream);
+
 /* Number of kernels the library has launched through this object (for launch accounting). */
 int64_t buzz_launch_count(buzz_t ctx);
 

@@ -36,7 +36,7 @@ def exported_symbols() -> list[str]:
     """Every entry point include/buzz.h declares."""
     return ["buzz_workspace_bytes", "buzz_create", "buzz_destroy", "buzz_prefill", "buzz_decode_step",
             "buzz_decode_step_host", "buzz_decode_layers", "buzz_decode_layers_host", "buzz_evict", "buzz_export_state", "buzz_import_state",
-            "buzz_export_prefill_scores", "buzz_prefill_static",
+            "buzz_export_prefill_scores", "buzz_prefill_static", "buzz_selftest_wait_expiry",
             "buzz_status", "buzz_launch_count", "buzz_set_decode_cluster", "buzz_set_sampling", "buzz_error_string"]
 
 
@@ -78,6 +78,8 @@ def load_library(build_if_missing: bool = True):
     lib.buzz_import_state.argtypes = [vp, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp]
     lib.buzz_export_prefill_scores.restype = ci
     lib.buzz_export_prefill_scores.argtypes = [vp, ci, ci, vp]
+    lib.buzz_selftest_wait_expiry.restype = ci
+    lib.buzz_selftest_wait_expiry.argtypes = [vp, ci, vp]
     lib.buzz_status.restype = ci
     lib.buzz_status.argtypes = [vp, vp]
     lib.buzz_launch_count.restype = ctypes.c_int64
@@ -199,6 +201,10 @@ class Buzz:
     # -- inspection ------------------------------------------------------------------------
     def status(self, stream=None) -> int:
         return self._lib.buzz_status(self._h, _stream_ptr(stream))
+
+    def selftest_wait_expiry(self, polls=1024, stream=None):
+        """buzz_selftest_wait_expiry: lets one bounded on-device wait run out; status() then reports -4 once."""
+        _check(self._lib.buzz_selftest_wait_expiry(self._h, int(polls), _stream_ptr(stream)), "buzz_selftest_wait_expiry")
 
     def launch_count(self) -> int:
         return self._lib.buzz_launch_count(self._h)

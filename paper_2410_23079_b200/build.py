@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libbuzz.so")
-SOURCES = ["api.cu", "decode.cu", "decode_bf16.cu", "evict.cu", "prefill_simt.cu", "prefill_tc.cu", "prefill_fill.cu", "prefill_noalloc.cu"]
+SOURCES = ["api.cu", "decode.cu", "decode_bf16.cu", "evict.cu", "prefill_simt.cu", "prefill_tc.cu", "prefill_fill.cu", "prefill_noalloc.cu", "selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--use_fast_math", "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

@@ -205,6 +205,21 @@ def test_overflow_status(cuda_device):
     bz.close()
 
 
+def test_bounded_wait_expiry_is_reported_and_survivable(cuda_device):
+    """A bounded on-device wait that nobody satisfies gives up by itself: the kernel ends, the status
+    word reports BUZZ_ERR_TIMEOUT once, and the same object then runs a normal prefill + decode +
+    evict to the oracle's result."""
+    w = workloads.scaled(workloads.get("C2"), layers=1, batch=1, q_heads=2, kv_heads=2, prompt_min=300,
+                         prompt_max=300, decode_steps=30, window=32, budget=96)
+    bz = make_buzz(w)
+    bz.selftest_wait_expiry(1024)
+    assert bz.status() == -4                           # BUZZ_ERR_TIMEOUT
+    assert bz.status() == 0                            # reading clears it
+    stats = run_lockstep(w, [(0, 0, 1)], bz=bz)        # the context and the object are intact
+    assert stats["evictions"] >= 1 and bz.status() == 0
+    bz.close()
+
+
 def test_no_progress_status(cuda_device):
     """segment = 2 gives s_hat = 1: a cache full of old tokens cannot shrink; reported, not looped."""
     w = workloads.scaled(workloads.get("C1"), sink=1, window=2, segment=2, hitters=1, budget=8,
