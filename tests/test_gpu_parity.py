@@ -65,8 +65,8 @@ def test_logn_scaling(cuda_device):
                 window=64, budget=180), [(0, 0, 0), (1, 1, 3)]),
     ("C4", dict(layers=1, batch=2, q_heads=8, kv_heads=2, prompt_min=900, prompt_max=900, decode_steps=130,
                 window=64, budget=300), [(0, 1, 0), (0, 0, 1)]),
-    ("C5", dict(layers=1, batch=3, q_heads=2, kv_heads=2, prompt_min=130, prompt_max=600, decode_steps=60,
-                window=48, budget=200), [(0, 0, 0), (0, 1, 1), (0, 2, 0)]),
+    ("C5", dict(layers=1, batch=3, q_heads=2, kv_heads=2, prompt_min=130, prompt_max=600, decode_steps=90,
+                window=48, budget=120), [(0, 0, 0), (0, 1, 1), (0, 2, 0)]),
 ])
 def test_logn_scaling_on_the_tensor_core_path(cuda_device, name, over, samples):
     """log_512(n) scaling on bf16, d = 128: the TMA/tcgen05 prefill kernels (prompts of several key
