@@ -1,9 +1,11 @@
 /* libbuzz -- C ABI of the BUZZ sparse KV-cache hot path on one NVIDIA B200 (sm_100a).
  *
- * BUZZ (arXiv 2410.23079) keeps, per attention head, a bounded KV cache laid out in position
- * order as  [ sink | old | new | window ]  (Algorithm 1): the first `sink` tokens, survivors of
+ * BUZZ (arXiv 2410.23079) keeps, per attention head, a bounded KV cache made of four parts, in
+ * position order  [ sink | old | new | window ]  (Algorithm 1): the first `sink` tokens, survivors of
  * earlier evictions ("old"), tokens that left the sliding window since the last eviction ("new"),
- * and the last `window` tokens. Each retained token carries an accumulated attention score
+ * and the last `window` tokens. (In device memory the window is a ring that sits right behind the
+ * sink, so that neither a decode step nor an eviction ever moves it; every call that hands cache
+ * contents to the host returns them in position order.) Each retained token carries an accumulated attention score
  * (Algorithm 2's input A). When the cache is full, the new tokens are cut into segments of
  * `segment` tokens and the top-scoring `hitters` of each segment survive, while the old tokens are
  * thinned to every s_hat-th, s_hat = floor((segment+1)/2) (Section 3.3).
@@ -185,25 +187,35 @@ int buzz_decode_layers_host(buzz_t ctx, int count, const int* layers, const void
 /* BUZZ eviction (Algorithm 1's sampling line and final concatenation; Algorithm 2) for one layer,
  * or for all layers when layer = -1. Per instance, entirely on the device: nothing happens unless
  * n >= budget (threshold buffering, Section 3.3) and n > sink + window (Remark 1). Otherwise the
- * old region keeps offsets 0, s_hat, 2 s_hat, ...; the new region [sink + n_old, n - window) is
- * cut into segments of `segment` slots (a short last one allowed) and each keeps its top
- * min(hitters, length) slots by (score descending, position ascending), emitted in position order;
- * K, V, score and pos are compacted in place as sink | old' | new' | window; n_old becomes
- * |old'| + |new'|. Calling it after every decode step is the intended use. */
+ * old tokens keep offsets 0, s_hat, 2 s_hat, ...; the new tokens (everything that left the window
+ * since the last eviction) are cut into segments of `segment` tokens (a short last one allowed) and
+ * each keeps its top min(hitters, length) tokens by (score descending, position ascending), in
+ * position order; K, V, score and pos of the survivors are compacted in place (sink and window are
+ * not moved); n_old becomes |old'| + |new'|. Calling it after every decode step is the intended use;
+ * when the library knows that no cache of the requested layers can be full (their last operation
+ * was a prefill, an eviction, or a decode step in fused mode) the call returns without launching. */
 int buzz_evict(buzz_t ctx, int layer, void* stream);
+
+/* Fused mode (Section 3.3's buffering without a second launch). With on != 0 every decode step
+ * (buzz_decode_step, buzz_decode_layers and their host-buffer forms) checks, in the kernel's own
+ * tail, whether the step has filled an instance's cache (n >= budget) and if so runs that instance's
+ * eviction right there, exactly as buzz_evict would have on the next call. The caches are then never
+ * full between calls, buzz_evict has nothing to do (and launches nothing), and the state after each
+ * step is bit-identical to decode step + buzz_evict in the default mode. Default: off. */
+int buzz_set_fused_evict(buzz_t ctx, int on);
 
 /* Test/checkpoint getter for one instance. Synchronises `stream`-independent: it waits for the
  * device. Any output pointer may be NULL. pos_host/score_host receive n entries, k_host/v_host
- * n*d elements of the cache dtype, in slot order (= position order). Buffers must hold `budget`
- * entries. */
+ * n*d elements of the cache dtype, in position order (sink, old, new, window; the window ring is
+ * un-rotated). Buffers must hold `budget` entries. */
 int buzz_export_state(buzz_t ctx, int layer, int seq, int kv_head, int32_t* n, int32_t* n_old,
                       int32_t* total_len, int32_t* pos_host, float* score_host, void* k_host,
                       void* v_host);
 
 /* The inverse of buzz_export_state (checkpoint restore, and how tests plant a cache state): loads
- * n slots (n <= budget, n_old <= n, total_len >= n) of one instance from host buffers laid out as
- * buzz_export_state writes them, and marks sequences 0..seq of the layer active. Waits for the
- * device before and after copying. */
+ * n tokens (n <= budget, n_old <= max(n - sink - window, 0), total_len >= n) of one instance from
+ * host buffers in position order, as buzz_export_state writes them, and marks sequences 0..seq of
+ * the layer active. Waits for the device before and after copying. */
 int buzz_import_state(buzz_t ctx, int layer, int seq, int kv_head, int32_t n, int32_t n_old,
                       int32_t total_len, const int32_t* pos_host, const float* score_host,
                       const void* k_host, const void* v_host);

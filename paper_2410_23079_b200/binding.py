@@ -37,7 +37,8 @@ def exported_symbols() -> list[str]:
     return ["buzz_workspace_bytes", "buzz_create", "buzz_destroy", "buzz_prefill", "buzz_decode_step",
             "buzz_decode_step_host", "buzz_decode_layers", "buzz_decode_layers_host", "buzz_evict", "buzz_export_state", "buzz_import_state",
             "buzz_export_prefill_scores", "buzz_prefill_static", "buzz_selftest_wait_expiry",
-            "buzz_status", "buzz_launch_count", "buzz_set_decode_cluster", "buzz_set_sampling", "buzz_error_string"]
+            "buzz_status", "buzz_launch_count", "buzz_set_decode_cluster", "buzz_set_sampling", "buzz_set_fused_evict",
+            "buzz_error_string"]
 
 
 def load_library(build_if_missing: bool = True):
@@ -86,6 +87,8 @@ def load_library(build_if_missing: bool = True):
     lib.buzz_launch_count.argtypes = [vp]
     lib.buzz_set_sampling.restype = ci
     lib.buzz_set_sampling.argtypes = [vp, ci, ci, ci]
+    lib.buzz_set_fused_evict.restype = ci
+    lib.buzz_set_fused_evict.argtypes = [vp, ci]
     lib.buzz_set_decode_cluster.restype = ci
     lib.buzz_set_decode_cluster.argtypes = [vp, ci]
     lib.buzz_error_string.restype = ctypes.c_char_p
@@ -211,6 +214,10 @@ class Buzz:
 
     def set_sampling(self, interval_new: bool, new_stride: int, old_stride: int):
         _check(self._lib.buzz_set_sampling(self._h, int(bool(interval_new)), new_stride, old_stride), "buzz_set_sampling")
+
+    def set_fused_evict(self, on: bool):
+        """buzz_set_fused_evict: decode steps run the eviction of a cache they fill in their own tail."""
+        _check(self._lib.buzz_set_fused_evict(self._h, int(bool(on))), "buzz_set_fused_evict")
 
     def set_decode_cluster(self, cluster_size: int):
         _check(self._lib.buzz_set_decode_cluster(self._h, cluster_size), "buzz_set_decode_cluster")

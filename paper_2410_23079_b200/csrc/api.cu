@@ -20,7 +20,7 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-  size_t k, v, score, pos, n, n_old, total, status, state_bytes;
+  size_t k, v, score, pos, n, n_old, total, ring, status, state_bytes;
   size_t lse, pscore, stage, scratch_bytes, stage_q, stage_kv;
 };
 
@@ -53,6 +53,7 @@ Layout make_layout(const buzz_shape& s, int budget) {
   L.n = off; off = align_up(off + inst * sizeof(int32_t));
   L.n_old = off; off = align_up(off + inst * sizeof(int32_t));
   L.total = off; off = align_up(off + inst * sizeof(int32_t));
+  L.ring = off; off = align_up(off + inst * sizeof(int32_t));
   L.status = off; off = align_up(off + 4 * sizeof(int32_t));
   L.state_bytes = off;
   off = 0;
@@ -124,6 +125,7 @@ int buzz_create(buzz_t* out, int sink, int window, int segment, int hitters, int
   c->st.n = reinterpret_cast<int32_t*>(sb + L.n);
   c->st.n_old = reinterpret_cast<int32_t*>(sb + L.n_old);
   c->st.total = reinterpret_cast<int32_t*>(sb + L.total);
+  c->st.ring = reinterpret_cast<int32_t*>(sb + L.ring);
   c->st.status = reinterpret_cast<int32_t*>(sb + L.status);
   char* sc = static_cast<char*>(scratch_dev);
   c->lse = reinterpret_cast<float*>(sc + L.lse);
@@ -133,6 +135,8 @@ int buzz_create(buzz_t* out, int sink, int window, int segment, int hitters, int
   c->stage_q = L.stage_q;
   c->stage_kv = L.stage_kv;
   c->batch = static_cast<int*>(calloc(shape->layers, sizeof(int)));
+  c->maybe_full = static_cast<char*>(calloc(shape->layers, 1));
+  c->fused_evict = 0;
   c->decode_cluster = 0;
   c->sm_count = 148;
   {
@@ -145,9 +149,10 @@ int buzz_create(buzz_t* out, int sink, int window, int segment, int hitters, int
   }
   c->launches = 0;
   c->last_kind = 0; c->last_layer = -1; c->last_stream = nullptr;
-  if (!c->batch) { delete c; return BUZZ_ERR_INVALID; }
+  if (!c->batch || !c->maybe_full) { free(c->batch); free(c->maybe_full); delete c; return BUZZ_ERR_INVALID; }
   if (cudaMemset(state_dev, 0, L.state_bytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
     free(c->batch);
+    free(c->maybe_full);
     delete c;
     return BUZZ_ERR_CUDA;
   }
@@ -158,6 +163,7 @@ int buzz_create(buzz_t* out, int sink, int window, int segment, int hitters, int
 void buzz_destroy(buzz_t c) {
   if (!c) return;
   free(c->batch);
+  free(c->maybe_full);
   delete c;
 }
 
@@ -180,6 +186,7 @@ int buzz_prefill(buzz_t c, int layer, const void* q, const void* k, const void* 
   if (e != cudaSuccess) return BUZZ_ERR_CUDA;
   c->batch[layer] = batch;
   e = buzz_launch_prefill_fill(c, layer, k, v, cu_seqlens_dev, batch, max_seqlen, s);
+  c->maybe_full[layer] = 0;   // the sampling rounds leave every sequence below its budget
   return e == cudaSuccess ? BUZZ_OK : BUZZ_ERR_CUDA;
 }
 
@@ -233,6 +240,24 @@ int buzz_decode_step_host(buzz_t c, int layer, const void* q_host, const void* k
 }
 
 namespace {
+// Position order <-> slot order of one instance ([sink | window ring | middle], cache_ops.cuh): the
+// retained tokens in position order are at most four contiguous runs of slots.
+struct Run { int first_out, first_slot, count; };
+int position_runs(const BuzzPolicy& pol, int n, int head, Run (&runs)[4]) {
+  const int k = pol.sink, w = pol.window;
+  int r = 0;
+  if (n <= k + w) {                       // ring still filling: slots are in position order
+    if (n > 0) runs[r++] = Run{0, 0, n};
+    return r;
+  }
+  const int m = n - k - w;
+  if (k > 0) runs[r++] = Run{0, 0, k};
+  runs[r++] = Run{k, k + w, m};
+  runs[r++] = Run{k + m, k + head, w - head};
+  if (head > 0) runs[r++] = Run{k + m + w - head, k, head};
+  return r;
+}
+
 // layers of one multi-layer call: in range, prefilled or empty, and pairwise distinct
 bool layers_ok(buzz_t c, int count, const int* layers) {
   if (!c || !layers || count < 1 || count > c->sh.layers) return false;
@@ -314,9 +339,22 @@ int buzz_decode_layers_host(buzz_t c, int count, const int* layers, const void* 
 
 int buzz_evict(buzz_t c, int layer, void* stream) {
   if (!c || layer < -1 || layer >= c->sh.layers) return BUZZ_ERR_INVALID;
-  cudaError_t e = layer < 0 ? buzz_launch_evict(c, 0, c->sh.layers, static_cast<cudaStream_t>(stream))
-                            : buzz_launch_evict(c, layer, 1, static_cast<cudaStream_t>(stream));
-  return e == cudaSuccess ? BUZZ_OK : BUZZ_ERR_CUDA;
+  // Layers whose caches are all known to be below their budget (a prefill, a fused decode step or an
+  // eviction was the last thing done to them) need no launch: the device predicate would find nothing.
+  const int begin = layer < 0 ? 0 : layer, count = layer < 0 ? c->sh.layers : 1;
+  bool due = false;
+  for (int l = begin; l < begin + count; ++l) due = due || c->maybe_full[l];
+  if (!due) return BUZZ_OK;
+  cudaError_t e = buzz_launch_evict(c, begin, count, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return BUZZ_ERR_CUDA;
+  for (int l = begin; l < begin + count; ++l) c->maybe_full[l] = 0;
+  return BUZZ_OK;
+}
+
+int buzz_set_fused_evict(buzz_t c, int on) {
+  if (!c) return BUZZ_ERR_INVALID;
+  c->fused_evict = on ? 1 : 0;
+  return BUZZ_OK;
 }
 
 int buzz_export_state(buzz_t c, int layer, int seq, int kv_head, int32_t* n, int32_t* n_old,
@@ -327,22 +365,26 @@ int buzz_export_state(buzz_t c, int layer, int seq, int kv_head, int32_t* n, int
     return BUZZ_ERR_INVALID;
   if (cudaDeviceSynchronize() != cudaSuccess) return BUZZ_ERR_CUDA;
   const size_t inst = buzz_inst(c->sh, layer, seq, kv_head);
-  int32_t cnt[3];
+  int32_t cnt[4];
   if (cudaMemcpy(&cnt[0], c->st.n + inst, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
   if (cudaMemcpy(&cnt[1], c->st.n_old + inst, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
   if (cudaMemcpy(&cnt[2], c->st.total + inst, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (cudaMemcpy(&cnt[3], c->st.ring + inst, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
   if (n) *n = cnt[0];
   if (n_old) *n_old = cnt[1];
   if (total_len) *total_len = cnt[2];
   const int m = cnt[0];
-  if (m < 0 || m > c->pol.budget) return BUZZ_ERR_INVALID;
+  if (m < 0 || m > c->pol.budget || cnt[3] < 0 || cnt[3] >= c->pol.window) return BUZZ_ERR_INVALID;
   const size_t row = (size_t)c->sh.head_dim * c->esize;
   const size_t slot0 = inst * c->pol.budget;
-  if (m > 0) {
-    if (pos_host && cudaMemcpy(pos_host, c->st.pos + slot0, (size_t)m * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
-    if (score_host && cudaMemcpy(score_host, c->st.score + slot0, (size_t)m * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
-    if (k_host && cudaMemcpy(k_host, c->st.K + slot0 * row, m * row, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
-    if (v_host && cudaMemcpy(v_host, c->st.V + slot0 * row, m * row, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
+  Run runs[4];
+  const int nr = position_runs(c->pol, m, cnt[3], runs);
+  for (int r = 0; r < nr; ++r) {           // the window ring is un-rotated: the output is in position order
+    const size_t o = runs[r].first_out, sl = slot0 + runs[r].first_slot, len = runs[r].count;
+    if (pos_host && cudaMemcpy(pos_host + o, c->st.pos + sl, len * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (score_host && cudaMemcpy(score_host + o, c->st.score + sl, len * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (k_host && cudaMemcpy(static_cast<char*>(k_host) + o * row, c->st.K + sl * row, len * row, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (v_host && cudaMemcpy(static_cast<char*>(v_host) + o * row, c->st.V + sl * row, len * row, cudaMemcpyDeviceToHost) != cudaSuccess) return BUZZ_ERR_CUDA;
   }
   return BUZZ_OK;
 }
@@ -353,23 +395,29 @@ int buzz_import_state(buzz_t c, int layer, int seq, int kv_head, int32_t n, int3
   if (!c || layer < 0 || layer >= c->sh.layers || seq < 0 || seq >= c->sh.max_batch || kv_head < 0 ||
       kv_head >= c->sh.kv_heads)
     return BUZZ_ERR_INVALID;
-  if (n < 0 || n > c->pol.budget || n_old < 0 || n_old > n || total_len < n) return BUZZ_ERR_INVALID;
+  if (n < 0 || n > c->pol.budget || n_old < 0 || total_len < n) return BUZZ_ERR_INVALID;
+  if (n_old > (n > c->pol.sink + c->pol.window ? n - c->pol.sink - c->pol.window : 0)) return BUZZ_ERR_INVALID;
   if (n > 0 && (!pos_host || !score_host || !k_host || !v_host)) return BUZZ_ERR_INVALID;
   if (cudaDeviceSynchronize() != cudaSuccess) return BUZZ_ERR_CUDA;
   const size_t inst = buzz_inst(c->sh, layer, seq, kv_head);
   const size_t row = (size_t)c->sh.head_dim * c->esize;
   const size_t slot0 = inst * c->pol.budget;
-  if (n > 0) {
-    if (cudaMemcpy(c->st.pos + slot0, pos_host, (size_t)n * 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
-    if (cudaMemcpy(c->st.score + slot0, score_host, (size_t)n * 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
-    if (cudaMemcpy(c->st.K + slot0 * row, k_host, n * row, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
-    if (cudaMemcpy(c->st.V + slot0 * row, v_host, n * row, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
+  Run runs[4];
+  const int nr = position_runs(c->pol, n, 0, runs);      // the window goes into the ring in order, head 0
+  for (int r = 0; r < nr; ++r) {
+    const size_t o = runs[r].first_out, sl = slot0 + runs[r].first_slot, len = runs[r].count;
+    if (cudaMemcpy(c->st.pos + sl, pos_host + o, len * 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (cudaMemcpy(c->st.score + sl, score_host + o, len * 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (cudaMemcpy(c->st.K + sl * row, static_cast<const char*>(k_host) + o * row, len * row, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
+    if (cudaMemcpy(c->st.V + sl * row, static_cast<const char*>(v_host) + o * row, len * row, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
   }
-  const int32_t cnt[3] = {n, n_old, total_len};
+  const int32_t cnt[4] = {n, n_old, total_len, 0};
   if (cudaMemcpy(c->st.n + inst, &cnt[0], 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
   if (cudaMemcpy(c->st.n_old + inst, &cnt[1], 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
   if (cudaMemcpy(c->st.total + inst, &cnt[2], 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
+  if (cudaMemcpy(c->st.ring + inst, &cnt[3], 4, cudaMemcpyHostToDevice) != cudaSuccess) return BUZZ_ERR_CUDA;
   if (c->batch[layer] < seq + 1) c->batch[layer] = seq + 1;
+  c->maybe_full[layer] = 1;
   c->last_kind = 2;
   return BUZZ_OK;
 }

@@ -20,14 +20,16 @@ struct BuzzPolicy {
 };
 
 // Device view of the persistent state. Instance index = ((layer * max_batch) + seq) * kv_heads + head.
+// Slot layout of an instance: [sink | window ring | middle (old, then new)], see cache_ops.cuh.
 struct BuzzState {
   char* K;            // [inst][budget][d] elements
   char* V;            // [inst][budget][d] elements
   float* score;       // [inst][budget]
   int32_t* pos;       // [inst][budget]
   int32_t* n;         // [inst] retained slots
-  int32_t* n_old;     // [inst] slots between sink and window that survived an eviction
+  int32_t* n_old;     // [inst] middle slots that survived an eviction
   int32_t* total;     // [inst] tokens seen so far (next position)
+  int32_t* ring;      // [inst] ring index of the oldest window token (0 while the ring is filling)
   int32_t* status;    // [4]: first error code, instance, detail, spare
 };
 
@@ -47,6 +49,8 @@ struct buzz_ctx {
   int* batch;         // active sequences per layer (host array)
   int decode_cluster; // 0 = choose automatically
   int sm_count;       // multiprocessors of the device that was current at buzz_create
+  int fused_evict;    // 1: a decode step runs the eviction of an instance that it fills, in its own tail
+  char* maybe_full;   // per layer (host): 1 if some cache of the layer may hold >= budget slots
   long long launches;
   // what the library launched last through this object (0 nothing, 1 a bf16 decode step, 2 anything else)
   int last_kind, last_layer;

@@ -1,0 +1,189 @@
+// Device-side operations on one instance's cache that more than one kernel needs: where an appended
+// token goes (Eq. 2 of the paper), and the BUZZ eviction of one instance (Algorithm 1's sampling
+// line and concatenation, Algorithm 2). Not part of the public ABI.
+//
+// Slot layout of an instance (budget slots, of which [0, n) are occupied):
+//   [0, sink)                    the first `sink` tokens                        (attention sink)
+//   [sink, sink + window)        the last `window` tokens, kept as a RING: ring index `head` holds the
+//                                oldest of them once the ring is full; while it is filling, tokens sit
+//                                at ring indices 0, 1, ... in order and head is 0
+//   [sink + window, n)           the middle region in position order: n_old survivors of earlier
+//                                evictions ("old"), then the tokens that have left the window since
+//                                the last eviction ("new")
+// Appending a token to a full ring replaces the oldest window token, which moves to slot n (the end
+// of the new tokens); an eviction therefore rewrites the middle region only and never moves the
+// window or the sink. Position order of the retained tokens is sink, middle, ring from `head` on.
+#pragma once
+
+#include "buzz_internal.cuh"
+
+namespace buzz_dev {
+
+__host__ __device__ inline int middle_begin(const BuzzPolicy& p) { return p.sink + p.window; }
+
+// Where the token appended at this step goes. slot_moved >= 0: the ring is full, the oldest window
+// token leaves slot_new for slot_moved (= n0) first.
+struct AppendPlan {
+  int slot_new;
+  int slot_moved;
+  int head_next;
+};
+__device__ inline AppendPlan plan_append(const BuzzPolicy& pol, int n0, int head) {
+  AppendPlan a;
+  if (n0 < pol.sink + pol.window) {
+    a.slot_new = n0; a.slot_moved = -1; a.head_next = head;
+  } else {
+    a.slot_new = pol.sink + head; a.slot_moved = n0; a.head_next = (head + 1 == pol.window) ? 0 : head + 1;
+  }
+  return a;
+}
+
+// Writes the appended token's K and V rows and position (and moves the token that leaves the window,
+// if any: its K, V and position; its score travels with the score update of the step). Called by
+// threads 0 .. 2*LPR of ONE CTA after every reader of the old rows is done. LPR = 16-byte lanes per row.
+template <int LPR>
+__device__ inline void append_rows(const BuzzState& st, const BuzzPolicy& pol, size_t inst, const AppendPlan& a,
+                                   int tot, const uint4* __restrict__ knew, const uint4* __restrict__ vnew, int tid) {
+  uint4* Kc = reinterpret_cast<uint4*>(st.K) + inst * (size_t)pol.budget * LPR;
+  uint4* Vc = reinterpret_cast<uint4*>(st.V) + inst * (size_t)pol.budget * LPR;
+  int32_t* pos = st.pos + inst * pol.budget;
+  if (tid < LPR) {
+    if (a.slot_moved >= 0) Kc[(size_t)a.slot_moved * LPR + tid] = Kc[(size_t)a.slot_new * LPR + tid];
+    Kc[(size_t)a.slot_new * LPR + tid] = knew[tid];
+  } else if (tid < 2 * LPR) {
+    const int t = tid - LPR;
+    if (a.slot_moved >= 0) Vc[(size_t)a.slot_moved * LPR + t] = Vc[(size_t)a.slot_new * LPR + t];
+    Vc[(size_t)a.slot_new * LPR + t] = vnew[t];
+  } else if (tid == 2 * LPR) {
+    if (a.slot_moved >= 0) pos[a.slot_moved] = pos[a.slot_new];
+    pos[a.slot_new] = tot;
+  }
+}
+
+struct Cand {
+  float v;
+  int idx;   // slot index, -1 = none
+};
+__device__ inline Cand better(Cand a, Cand b) {
+  // The winner is the larger score; equal scores go to the lower slot (= lower position).
+  if (a.idx < 0) return b;
+  if (b.idx < 0) return a;
+  if (b.v > a.v || (b.v == a.v && b.idx < a.idx)) return b;
+  return a;
+}
+
+// One eviction of one instance by one whole CTA of THREADS threads (all of them must call it; the
+// trigger n >= budget and Remark 1's n > sink + window are the caller's to check).
+//   old region  [mb, mb + n_old)   keep offsets 0, s_hat, 2 s_hat, ...          (interval sampling)
+//   new region  [mb + n_old, n)    per segment of s slots keep the top-h by (score desc, position asc),
+//                                  in position order                            (Algorithm 2)
+// with mb = sink + window. The counts depend only on n and n_old, so every destination is closed-form;
+// only the winners inside a segment depend on the scores. A warp owns a segment: each lane holds the
+// candidates lane, lane+32, ...; h rounds of a shuffle arg-max flag the winners, ballots + popcounts
+// give their rank in position order. Compaction is an in-place stable left shift (destination <=
+// source): ascending chunks, a chunk's sources read into registers, a barrier, then the writes.
+// `src` is shared memory for at least kept_old + kept_new ints (never more than n - sink - window).
+template <int ROW_BYTES, int THREADS>
+__device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_t inst, int n, int n_old,
+                               int32_t* src) {
+  constexpr int kRowsPerPass = 4;   // rows of K and of V each 16-byte lane moves per pass
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int s = pol.segment, h = pol.hitters, s_hat = pol.s_hat;
+  const int mb = middle_begin(pol);
+  const int new_begin = mb + n_old;
+  const int n_new = n - new_begin;
+  const int kept_old = (n_old + s_hat - 1) / s_hat;
+  const int nseg = (n_new + s - 1) / s;
+  const int last_len = n_new - (nseg - 1) * s;
+  const int kept_new = nseg > 0 ? (nseg - 1) * h + min(h, last_len) : 0;
+  const int kept_mid = kept_old + kept_new;
+
+  float* score = st.score + inst * pol.budget;
+  int32_t* pos = st.pos + inst * pol.budget;
+
+  // ---- selection: src[t] = source slot of middle destination mb + t ---------------------------
+  for (int t = tid; t < kept_old; t += THREADS) src[t] = mb + t * s_hat;
+  for (int seg = warp; seg < nseg; seg += THREADS / 32) {
+    const int lo = new_begin + seg * s;
+    const int len = min(s, n - lo);
+    const int want = min(h, len);
+    const int out0 = kept_old + seg * h;
+    if (pol.interval_new) {                         // ablation: the first `want` slots of the segment
+      for (int r = lane; r < want; r += 32) src[out0 + r] = lo + r;
+      continue;
+    }
+    unsigned chosen = 0;                            // bit i: candidate lo + i*32 + lane is a winner
+    for (int r = 0; r < want; ++r) {
+      Cand best{0.f, -1};
+      for (int i = 0, j = lane; j < len; ++i, j += 32) {
+        if (chosen >> i & 1u) continue;
+        best = better(best, Cand{score[lo + j], lo + j});
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        Cand o;
+        o.v = __shfl_xor_sync(0xffffffffu, best.v, off);
+        o.idx = __shfl_xor_sync(0xffffffffu, best.idx, off);
+        best = better(best, o);
+      }
+      const int w = best.idx - lo;
+      if ((w & 31) == lane) chosen |= 1u << (w >> 5);
+    }
+    int before = 0;                                 // winners at lower positions
+    for (int i = 0; i * 32 < len; ++i) {
+      const bool mine = chosen >> i & 1u;
+      const unsigned b = __ballot_sync(0xffffffffu, mine);
+      if (mine) src[out0 + before + __popc(b & ((1u << lane) - 1u))] = lo + i * 32 + lane;
+      before += __popc(b);
+    }
+  }
+  __syncthreads();
+
+  // ---- compaction of score and pos ------------------------------------------------------------
+  for (int base = 0; base < kept_mid; base += THREADS) {
+    const int t = base + tid;
+    float sc = 0.f;
+    int32_t ps = 0;
+    if (t < kept_mid) { sc = score[src[t]]; ps = pos[src[t]]; }
+    __syncthreads();
+    if (t < kept_mid) { score[mb + t] = sc; pos[mb + t] = ps; }
+  }
+
+  // ---- compaction of the K and V rows ---------------------------------------------------------
+  constexpr int LPR = ROW_BYTES / 16;               // 16-byte lanes per row
+  constexpr int ROWS = THREADS / LPR * kRowsPerPass;
+  uint4* Kc = reinterpret_cast<uint4*>(st.K + inst * (size_t)pol.budget * ROW_BYTES);
+  uint4* Vc = reinterpret_cast<uint4*>(st.V + inst * (size_t)pol.budget * ROW_BYTES);
+  const int sub = tid % LPR, rgrp = tid / LPR;
+  // The first old survivor stays where it is.
+  for (int base = kept_old > 0 ? 1 : 0; base < kept_mid; base += ROWS) {
+    uint4 kr[kRowsPerPass], vr[kRowsPerPass];
+#pragma unroll
+    for (int u = 0; u < kRowsPerPass; ++u) {
+      const int t = base + u * (THREADS / LPR) + rgrp;
+      if (t < kept_mid) {
+        const int sj = src[t];
+        kr[u] = Kc[(size_t)sj * LPR + sub];
+        vr[u] = Vc[(size_t)sj * LPR + sub];
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < kRowsPerPass; ++u) {
+      const int t = base + u * (THREADS / LPR) + rgrp;
+      if (t < kept_mid) {
+        Kc[(size_t)(mb + t) * LPR + sub] = kr[u];
+        Vc[(size_t)(mb + t) * LPR + sub] = vr[u];
+      }
+    }
+  }
+
+  if (tid == 0) {
+    const int n2 = mb + kept_mid;
+    st.n[inst] = n2;
+    st.n_old[inst] = kept_mid;
+    if (n2 >= pol.budget) buzz_set_status(st.status, BUZZ_ERR_NO_PROGRESS, (int)inst, n2);
+  }
+}
+
+}  // namespace buzz_dev

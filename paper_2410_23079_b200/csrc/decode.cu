@@ -13,11 +13,13 @@
 //            memory, derives the global normaliser, adds the now-exact probabilities of ITS chunk
 //            to the scores, and CTA 0 merges the partial outputs.
 // Nothing is staged in global memory and every reduction has a fixed order, so the result is
-// deterministic. The appended token's row is read from k_new/v_new rather than from the cache slot
-// the same kernel writes.
+// deterministic. The appended token's row is read from k_new/v_new throughout and stored after the
+// cluster barrier: into the window ring, whose oldest token first moves to the end of the middle
+// region (cache_ops.cuh). In fused mode CTA 0 then runs the instance's eviction if the step filled
+// the cache.
 #include <cooperative_groups.h>
 
-#include "buzz_internal.cuh"
+#include "cache_ops.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -63,7 +65,7 @@ template <typename T, int D, int G>
 __global__ void __launch_bounds__(kThreads)
 decode_kernel(BuzzState st, BuzzPolicy pol, const T* __restrict__ q, const T* __restrict__ k_new,
               const T* __restrict__ v_new, T* __restrict__ out, int layer, int max_batch,
-              int kv_heads, int chunk_cap, float scale_log2, int logn) {
+              int kv_heads, int chunk_cap, float scale_log2, int logn, int fused_evict) {
   constexpr int EPL = Vec16<T>::N;              // elements per 16-byte lane
   constexpr int LPR = D / EPL;                  // lanes per row
   constexpr int RPW = 32 / LPR;                 // rows per warp-wide load
@@ -85,9 +87,11 @@ decode_kernel(BuzzState st, BuzzPolicy pol, const T* __restrict__ q, const T* __
   float* invL = fr + kMaxCluster * G;                        // [G]
   float* owarp = invL + G;                                   // [kWarps][G][D]
   float* sl = owarp + kWarps * G * D;                        // [G][chunk_cap]
+  int32_t* evict_src = reinterpret_cast<int32_t*>(sl + (size_t)G * chunk_cap);   // fused mode: [budget - sink - window]
 
   const int n0 = st.n[inst];
   const int tot = st.total[inst];
+  const int ring_head = st.ring[inst];
   if (n0 >= pol.budget) {          // uniform over the cluster: every CTA read the same n0
     if (rank == 0 && tid == 0) buzz_set_status(st.status, BUZZ_ERR_OVERFLOW, (int)inst, n0);
     return;
@@ -106,12 +110,10 @@ decode_kernel(BuzzState st, BuzzPolicy pol, const T* __restrict__ q, const T* __
   const uint4* knew = reinterpret_cast<const uint4*>(k_new) + ((size_t)seq * kv_heads + head) * LPR;
   const uint4* vnew = reinterpret_cast<const uint4*>(v_new) + ((size_t)seq * kv_heads + head) * LPR;
 
-  // The CTA whose chunk holds slot n0 stores the appended token (Eq. 2).
-  if (n0 >= lo && n0 < hi) {
-    if (tid < LPR) (reinterpret_cast<uint4*>(st.K) + cache_off)[(size_t)n0 * LPR + tid] = knew[tid];
-    else if (tid < 2 * LPR) (reinterpret_cast<uint4*>(st.V) + cache_off)[(size_t)n0 * LPR + tid - LPR] = vnew[tid - LPR];
-    else if (tid == 2 * LPR) st.pos[inst * pol.budget + n0] = tot;
-  }
+  // Logical slot n0 is the token being appended (Eq. 2): read from k_new / v_new throughout, stored
+  // after the cluster barrier (with a full window ring it replaces the oldest window token, whose
+  // row other CTAs are still reading until then).
+  const buzz_dev::AppendPlan app = buzz_dev::plan_append(pol, n0, ring_head);
 
   // ---- phase 1: logits ------------------------------------------------------------------
   float mx[G];
@@ -246,9 +248,13 @@ decode_kernel(BuzzState st, BuzzPolicy pol, const T* __restrict__ q, const T* __
 
   // ---- combine across the cluster -------------------------------------------------------
   cluster.sync();
-  if (rank == 0 && tid == 0) {       // every CTA has read n0/tot before the barrier
-    st.n[inst] = n1;
-    st.total[inst] = tot + 1;
+  if (rank == 0) {                   // every CTA has read n0/tot/ring and all old rows before the barrier
+    buzz_dev::append_rows<LPR>(st, pol, inst, app, tot, knew, vnew, tid);
+    if (tid == kThreads - 1) {
+      st.n[inst] = n1;
+      st.total[inst] = tot + 1;
+      st.ring[inst] = app.head_next;
+    }
   }
   if (tid < G) {
     float M = -INFINITY;
@@ -263,7 +269,11 @@ decode_kernel(BuzzState st, BuzzPolicy pol, const T* __restrict__ q, const T* __
     invL[tid] = 1.0f / L;
   }
   __syncthreads();
-  // scores of this CTA's chunk: += sum over the group's heads of the exact probabilities
+  // scores of this CTA's chunk: += sum over the group's heads of the exact probabilities. With a full
+  // ring the token leaving the window (still at slot app.slot_new) takes its score along to slot n0,
+  // and the appended token's first score lands in app.slot_new after the last barrier.
+  float pending_score = 0.f;
+  bool has_pending = false;
   {
     float* score = st.score + inst * pol.budget;
     for (int j = tid; j < cnt; j += kThreads) {
@@ -271,7 +281,14 @@ decode_kernel(BuzzState st, BuzzPolicy pol, const T* __restrict__ q, const T* __
 #pragma unroll
       for (int g = 0; g < G; ++g) add += sl[g * chunk_cap + j] * (fr[rank * G + g] * invL[g]);
       const int slot = lo + j;
-      score[slot] = (slot == n0 ? 0.f : score[slot]) + add;
+      if (slot == n0) {
+        if (app.slot_moved >= 0) { pending_score = add; has_pending = true; }
+        else score[n0] = add;
+      } else if (slot == app.slot_new) {             // only with a full ring: slot_new < n0
+        score[n0] = score[slot] + add;
+      } else {
+        score[slot] += add;
+      }
     }
   }
   if (rank == 0) {
@@ -284,6 +301,9 @@ decode_kernel(BuzzState st, BuzzPolicy pol, const T* __restrict__ q, const T* __
     }
   }
   cluster.sync();                    // peers may still be reading this CTA's shared memory
+  if (has_pending) st.score[inst * pol.budget + app.slot_new] = pending_score;
+  if (fused_evict && rank == 0 && n1 >= pol.budget && n1 > pol.sink + pol.window)
+    buzz_dev::evict_instance<D * (int)sizeof(T), kThreads>(st, pol, inst, n1, st.n_old[inst], evict_src);
 }
 
 template <typename T, int D, int G>
@@ -292,7 +312,8 @@ cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, con
   const int batch = c->batch[layer];
   const int chunk_cap = (c->pol.budget + cluster_size - 1) / cluster_size;
   const size_t smem = sizeof(Partial<G, D>) +
-                      sizeof(float) * (kWarps * G + kMaxCluster * G + G + kWarps * G * D + (size_t)G * chunk_cap);
+                      sizeof(float) * (kWarps * G + kMaxCluster * G + G + kWarps * G * D + (size_t)G * chunk_cap) +
+                      (c->fused_evict ? sizeof(int32_t) * (size_t)(c->pol.budget - c->pol.sink - c->pol.window) : 0);
   static BuzzSmemOptIn opt_in;
   if (cudaError_t e = opt_in.ensure(decode_kernel<T, D, G>, smem); e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
@@ -310,7 +331,7 @@ cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, con
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)D);
   return cudaLaunchKernelEx(&cfg, decode_kernel<T, D, G>, c->st, c->pol, (const T*)q, (const T*)k_new,
                             (const T*)v_new, (T*)out, layer, c->sh.max_batch, c->sh.kv_heads,
-                            chunk_cap, scale_log2, (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0);
+                            chunk_cap, scale_log2, (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0, c->fused_evict);
 }
 
 template <typename T, int D>
@@ -362,6 +383,9 @@ cudaError_t buzz_launch_decode(buzz_ctx* c, int layer, const void* q, const void
                               : launch_g<float, 64>(c, layer, q, k_new, v_new, out, cs, stream);
     c->last_kind = 2;
   }
-  if (e == cudaSuccess) c->launches += 1;
+  if (e == cudaSuccess) {
+    c->launches += 1;
+    c->maybe_full[layer] = c->fused_evict ? 0 : 1;   // a fused step leaves every cache below its budget
+  }
   return e;
 }

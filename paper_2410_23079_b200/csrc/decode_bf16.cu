@@ -19,9 +19,14 @@
 //   combine  as in decode.cu: partial (max, sum, output) per CTA in shared memory, one cluster
 //            barrier, exact probabilities of the CTA's own chunk added to the scores, CTA 0 writes
 //            the output. No global scratch, no atomics, fixed-order reductions.
+//   append   after the barrier (every reader of the old rows is done) CTA 0 stores the new token: into
+//            the window ring, whose oldest token first moves to the end of the middle region (see
+//            cache_ops.cuh); that token's score moves with the score update.
+//   evict    (fused mode) if the step filled the cache, CTA 0 runs the instance's eviction in the
+//            kernel's tail, so no separate eviction launch is needed.
 #include <cooperative_groups.h>
 
-#include "buzz_internal.cuh"
+#include "cache_ops.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -67,7 +72,7 @@ __global__ void __launch_bounds__(kThreads)
 decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict__ q,
                    const __nv_bfloat16* __restrict__ k_new, const __nv_bfloat16* __restrict__ v_new,
                    __nv_bfloat16* __restrict__ out, int layer, int max_batch, int kv_heads,
-                   int chunk_cap, float scale_log2, int logn, int mode, int next_layer) {
+                   int chunk_cap, float scale_log2, int logn, int mode, int next_layer, int fused_evict) {
   constexpr int NCH = D / 8;          // 16-byte chunks per row
   constexpr int KL = NCH / 4;         // K chunks per lane and row
   constexpr int VJ = NCH / 8;         // V chunks per lane and row
@@ -90,6 +95,7 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   float* invL = Mg + G;                                      // [G]
   float* owarp = invL + G;                                   // [kWarps][G][D]
   float* sl = owarp + kWarps * G * D;                        // [G][chunk_cap] logits (log2 domain)
+  int32_t* evict_src = reinterpret_cast<int32_t*>(sl + (size_t)G * chunk_cap);   // fused mode: [budget - sink - window]
 
   // Programmatic dependent launch; the host picks one of three modes.
   //   kWaitFirst  wait for everything earlier in the stream, then let the next launch begin.
@@ -117,6 +123,7 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   }
   const int n0 = st.n[inst];
   const int tot = st.total[inst];
+  const int ring_head = st.ring[inst];
   if (n0 >= pol.budget) {          // uniform over the cluster: every CTA read the same n0
     if (rank == 0 && tid == 0) buzz_set_status(st.status, BUZZ_ERR_OVERFLOW, (int)inst, n0);
     if (mode == kOverlap) asm volatile("griddepcontrol.wait;" ::: "memory");   // still finish after the member before
@@ -136,12 +143,10 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   const uint4* knew = reinterpret_cast<const uint4*>(k_new) + ((size_t)seq * kv_heads + head) * NCH;
   const uint4* vnew = reinterpret_cast<const uint4*>(v_new) + ((size_t)seq * kv_heads + head) * NCH;
 
-  // The CTA whose chunk holds slot n0 stores the appended token (Eq. 2).
-  if (n0 >= lo && n0 < hi) {
-    if (tid < NCH) (reinterpret_cast<uint4*>(st.K) + cache_off)[(size_t)n0 * NCH + tid] = knew[tid];
-    else if (tid < 2 * NCH) (reinterpret_cast<uint4*>(st.V) + cache_off)[(size_t)n0 * NCH + tid - NCH] = vnew[tid - NCH];
-    else if (tid == 2 * NCH) st.pos[inst * pol.budget + n0] = tot;
-  }
+  // Logical slot n0 is the token being appended (Eq. 2): it is read from k_new / v_new throughout and
+  // stored only after the cluster barrier below, because with a full window ring it replaces the
+  // oldest window token, whose row other CTAs are still reading until then.
+  const buzz_dev::AppendPlan app = buzz_dev::plan_append(pol, n0, ring_head);
 
   // Rolling L2 prefetch. The CTA's traffic is one stream: its K rows, then its V rows, then (as a
   // hint only) the head of the same chunk in the NEXT layer's K cache, which the next decode launch
@@ -325,9 +330,13 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   // ---- combine across the cluster -------------------------------------------------------
   cluster.sync();
   if (mode == kOverlap) asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (rank == 0 && tid == 0) {       // every CTA has read n0/tot before the barrier
-    st.n[inst] = n1;
-    st.total[inst] = tot + 1;
+  if (rank == 0) {                   // every CTA has read n0/tot/ring and all old rows before the barrier
+    buzz_dev::append_rows<NCH>(st, pol, inst, app, tot, knew, vnew, tid);
+    if (tid == kThreads - 1) {
+      st.n[inst] = n1;
+      st.total[inst] = tot + 1;
+      st.ring[inst] = app.head_next;
+    }
   }
   if (tid < G) {
     float M = -INFINITY;
@@ -343,7 +352,12 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
     invL[tid] = 1.0f / L;
   }
   __syncthreads();
-  // scores of this CTA's chunk: += sum over the group's heads of the exact fp32 probabilities
+  // scores of this CTA's chunk: += sum over the group's heads of the exact fp32 probabilities. With a
+  // full ring the token leaving the window (still at slot app.slot_new) takes its score along to slot
+  // n0, and the appended token's first score lands in app.slot_new -- stored only after the last
+  // barrier, once the thread that reads the old value there is done.
+  float pending_score = 0.f;
+  bool has_pending = false;
   {
     float* score = st.score + inst * pol.budget;
     for (int j = tid; j < cnt; j += kThreads) {
@@ -351,7 +365,14 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
 #pragma unroll
       for (int g = 0; g < G; ++g) add += exp2f(sl[g * chunk_cap + j] - Mg[g]) * invL[g];
       const int slot = lo + j;
-      score[slot] = (slot == n0 ? 0.f : score[slot]) + add;
+      if (slot == n0) {
+        if (app.slot_moved >= 0) { pending_score = add; has_pending = true; }
+        else score[n0] = add;
+      } else if (slot == app.slot_new) {             // only with a full ring: slot_new < n0
+        score[n0] = score[slot] + add;
+      } else {
+        score[slot] += add;
+      }
     }
   }
   if (rank == 0) {
@@ -364,6 +385,11 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
     }
   }
   cluster.sync();                    // peers may still be reading this CTA's shared memory
+  if (has_pending) st.score[inst * pol.budget + app.slot_new] = pending_score;
+  // Fused eviction (Algorithm 1's trigger: the cache is full after this step). Every score, row and
+  // counter of the instance was written before the barrier above, by this cluster.
+  if (fused_evict && rank == 0 && n1 >= pol.budget && n1 > pol.sink + pol.window)
+    buzz_dev::evict_instance<D * 2, kThreads>(st, pol, inst, n1, st.n_old[inst], evict_src);
 }
 
 template <int D, int G>
@@ -373,7 +399,8 @@ cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, con
   const int chunk_cap = (((c->pol.budget + cluster_size - 1) / cluster_size + 1) & ~1) + 2;
   const size_t smem = sizeof(Partial<G, D>) +
                       sizeof(float) * (kWarps * kHeads + kHeads + kMaxCluster * G + 2 * G +
-                                       kWarps * G * D + (size_t)G * chunk_cap);
+                                       kWarps * G * D + (size_t)G * chunk_cap) +
+                      (c->fused_evict ? sizeof(int32_t) * (size_t)(c->pol.budget - c->pol.sink - c->pol.window) : 0);
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
   static BuzzSmemOptIn opt_in;
   if (cudaError_t e = opt_in.ensure(decode_bf16_kernel<D, G>, smem); e != cudaSuccess) return e;
@@ -395,7 +422,7 @@ cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, con
   return cudaLaunchKernelEx(&cfg, decode_bf16_kernel<D, G>, c->st, c->pol, (const __nv_bfloat16*)q,
                             (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, (__nv_bfloat16*)out,
                             layer, c->sh.max_batch, c->sh.kv_heads, chunk_cap, scale_log2,
-                            (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0, mode, next_layer);
+                            (c->sh.flags & BUZZ_FLAG_LOGN) ? 1 : 0, mode, next_layer, c->fused_evict);
 }
 
 template <int D>

@@ -7,7 +7,9 @@
 // survivors. Counts never depend on the scores, so after R rounds the f-th middle survivor is
 // the (f * s_hat^(R-1))-th winner of round one: destination slots are closed-form and the gather
 // is embarrassingly parallel -- each 16-lane group resolves its own slot's source token (rescanning
-// one segment of <= s scores) and copies that row.
+// one segment of <= s scores) and copies that row. The cache is laid out [sink | window ring |
+// middle] (cache_ops.cuh): the prompt's last `window` tokens fill the ring in order (head 0) and
+// the survivors between sink and window follow it.
 #include "buzz_internal.cuh"
 
 namespace {
@@ -90,8 +92,9 @@ prefill_fill_kernel(BuzzState st, BuzzPolicy pol, const char* __restrict__ k, co
   if (blockIdx.x == 0 && tid == 0) {
     if (plan.error) {
       buzz_set_status(st.status, BUZZ_ERR_NO_PROGRESS, (int)inst, N);
-      st.n[inst] = 0; st.n_old[inst] = 0; st.total[inst] = N;
+      st.n[inst] = 0; st.n_old[inst] = 0; st.total[inst] = N; st.ring[inst] = 0;
     } else {
+      st.ring[inst] = 0;
       st.n[inst] = plan.n_final;
       st.n_old[inst] = plan.rounds > 0 ? plan.n_mid : 0;
       st.total[inst] = N;
@@ -105,13 +108,16 @@ prefill_fill_kernel(BuzzState st, BuzzPolicy pol, const char* __restrict__ k, co
     if (plan.rounds == 0 || t < pol.sink) src = t;
     else if (t < pol.sink + plan.n_mid) src = round_one_winner(sc, N, pol, (int)((t - pol.sink) * plan.stride));
     else src = N - pol.window + (t - pol.sink - plan.n_mid);
+    // t counts the survivors in position order; their slots: sink, then (behind the ring) the middle,
+    // and the last `window` tokens in the ring right after the sink
+    const int slot = t < pol.sink ? t : (t < pol.sink + plan.n_mid ? t + pol.window : t - plan.n_mid);
     const size_t g = ((size_t)(tok0 + src) * kv_heads + head) * LPR + sub;
-    const size_t d = (cache_row0 + t) * LPR + sub;
+    const size_t d = (cache_row0 + slot) * LPR + sub;
     reinterpret_cast<uint4*>(st.K)[d] = __ldg(reinterpret_cast<const uint4*>(k) + g);
     reinterpret_cast<uint4*>(st.V)[d] = __ldg(reinterpret_cast<const uint4*>(v) + g);
     if (sub == 0) {
-      st.score[cache_row0 + t] = sc[src];
-      st.pos[cache_row0 + t] = src;
+      st.score[cache_row0 + slot] = sc[src];
+      st.pos[cache_row0 + slot] = src;
     }
   }
 }

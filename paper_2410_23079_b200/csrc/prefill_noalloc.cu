@@ -83,6 +83,7 @@ extern "C" int buzz_prefill_static(buzz_t c, int layer, const void* q, const voi
   if (e != cudaSuccess) return BUZZ_ERR_CUDA;
   c->batch[layer] = batch;          // the host array is shared between `c` and the view
   e = buzz_launch_prefill_fill(&view, layer, k, v, cu_seqlens_dev, batch, max_seqlen, s);
+  c->maybe_full[layer] = 0;
   c->launches += launches + view.launches;
   c->last_kind = view.last_kind;     // bookkeeping the launches made on the view
   return e == cudaSuccess ? BUZZ_OK : BUZZ_ERR_CUDA;

@@ -97,6 +97,111 @@ def test_dtype_headdim_group_matrix(cuda_device, dtype, d, g):
     assert stats["evictions"] >= 2
 
 
+@pytest.mark.parametrize("name,over", [
+    ("C1", dict(prompt_min=3, prompt_max=3, decode_steps=230, sink=2, window=16, segment=4, budget=41)),
+    ("C2", dict(layers=1, batch=2, q_heads=2, kv_heads=2, prompt_min=9, prompt_max=9, decode_steps=260, sink=4,
+                window=24, segment=5, hitters=2, budget=64)),
+    ("C4", dict(layers=1, batch=1, q_heads=4, kv_heads=1, prompt_min=30, prompt_max=30, decode_steps=150, sink=0,
+                window=1, segment=3, budget=20)),
+])
+def test_window_ring_from_empty_to_many_rotations(cuda_device, name, over):
+    """The window lives in a ring behind the sink. Starting from a prompt shorter than sink + window,
+    the ring first fills in order, then every step replaces its oldest token (which moves to the end
+    of the middle region, score and position included), and evictions compact the middle only. The
+    ring goes round many times here; every step and every eviction is checked against the oracle,
+    whose cache is in plain position order. Also the degenerate ring of one slot with no sink."""
+    w = workloads.scaled(workloads.get(name), **over)
+    samples = [(0, b, w.kv_heads - 1) for b in range(w.batch)]
+    stats = run_lockstep(w, samples, check_every=1)
+    assert stats["evictions"] >= 8
+
+
+def test_export_import_round_trip_with_a_rotated_ring(cuda_device):
+    """A cache exported mid-run (ring head somewhere in the middle) and imported into a fresh object
+    continues to the same results: the exported arrays are in position order whatever the ring's
+    phase. (The import restarts the ring at head 0, so the slot order, and with it the fp32 summation
+    order, differs between the two objects: outputs and scores agree to rounding, not bit for bit.)"""
+    w = workloads.scaled(workloads.get("C2"), layers=1, batch=1, q_heads=2, kv_heads=2, prompt_min=200,
+                         prompt_max=200, decode_steps=120, window=32, budget=100)
+    a, b = make_buzz(w), make_buzz(w)
+    q, k, v, cu = workloads.prefill_inputs(w, 0, "cuda:0")
+    a.prefill(0, q, k, v, cu, 200, torch.empty_like(q))
+    qd, kd, vd = workloads.decode_inputs(w, 0, "cuda:0")
+    o = torch.empty_like(qd[0])
+    for t in range(45):                                 # 45 steps: the head is at ring index 13
+        a.decode_step(0, qd[t], kd[t], vd[t], o); a.evict(0)
+    for h in range(2):
+        st = a.export_state(0, 0, h)
+        assert torch.all(st["pos"][1:] > st["pos"][:-1])                       # position order
+        assert st["pos"][-32:].tolist() == list(range(245 - 32, 245))           # the window, un-rotated
+        b.import_state(0, 0, h, st["n_old"], st["total_len"], st["pos"], st["score"], st["k"], st["v"])
+    for t in range(45, w.decode_steps):
+        oa, ob = torch.empty_like(qd[t]), torch.empty_like(qd[t])
+        a.decode_step(0, qd[t], kd[t], vd[t], oa); a.evict(0)
+        b.decode_step(0, qd[t], kd[t], vd[t], ob); b.evict(0)
+        torch.testing.assert_close(oa.float(), ob.float(), atol=1e-2, rtol=1e-2)
+    for h in range(2):
+        x, y = a.export_state(0, 0, h), b.export_state(0, 0, h)
+        assert (x["n"], x["n_old"], x["total_len"]) == (y["n"], y["n_old"], y["total_len"])
+        for key in ("pos", "k", "v"):
+            assert torch.equal(x[key], y[key])
+        torch.testing.assert_close(x["score"], y["score"], atol=0.0, rtol=1e-4)
+    assert a.status() == 0 and b.status() == 0
+    a.close(); b.close()
+
+
+@pytest.mark.parametrize("name,over,layers_call", [
+    ("C2", dict(layers=3, batch=2, q_heads=4, kv_heads=4, prompt_min=300, prompt_max=300, decode_steps=160,
+                window=32, budget=100), False),
+    ("C4", dict(layers=2, batch=3, q_heads=8, kv_heads=2, prompt_min=150, prompt_max=420, decode_steps=140,
+                window=48, budget=150, segment=16, hitters=2), True),
+    ("C1", dict(layers=2, batch=2, q_heads=2, kv_heads=2, prompt_min=100, prompt_max=100, decode_steps=150,
+                window=16, budget=60), False),
+])
+def test_fused_eviction_matches_separate_calls(cuda_device, name, over, layers_call):
+    """Fused mode: a decode step that fills a cache evicts it in the kernel's own tail. Outputs of every
+    step and the final caches must equal, bit for bit, decode step + buzz_evict in the default mode
+    (which the lock-step tests check against the oracle); in fused mode buzz_evict launches nothing."""
+    w = workloads.scaled(workloads.get(name), **over)
+    lens = workloads.prompt_lengths(w)
+    pre, dec = _stack(w)
+    ref, fused = make_buzz(w), make_buzz(w)
+    fused.set_fused_evict(True)
+    for bz in (ref, fused):
+        for l in range(w.layers):
+            q, k, v, cu = pre[l]
+            bz.prefill(l, q, k, v, cu, max(lens), torch.empty_like(q))
+    L = list(range(w.layers))
+    evict_launches = 0
+    for t in range(w.decode_steps):
+        o_ref = [torch.empty_like(dec[l][0][t]) for l in L]
+        o_fus = [torch.empty_like(dec[l][0][t]) for l in L]
+        for bz, outs in ((ref, o_ref), (fused, o_fus)):
+            if layers_call:
+                bz.decode_layers(L, [dec[l][0][t] for l in L], [dec[l][1][t] for l in L], [dec[l][2][t] for l in L], outs)
+            else:
+                for l in L:
+                    bz.decode_step(l, dec[l][0][t], dec[l][1][t], dec[l][2][t], outs[l])
+        ref.evict(-1)
+        before = fused.launch_count()
+        fused.evict(-1 if t % 2 else 0)
+        evict_launches += fused.launch_count() - before
+        for l in L:
+            assert torch.equal(o_ref[l], o_fus[l]), f"step {t} layer {l}"
+    assert evict_launches == 0
+    evicted = False
+    for l in L:
+        for b in range(w.batch):
+            for h in range(w.kv_heads):
+                x, y = ref.export_state(l, b, h), fused.export_state(l, b, h)
+                assert (x["n"], x["n_old"], x["total_len"]) == (y["n"], y["n_old"], y["total_len"]), (l, b, h)
+                for key in ("pos", "score", "k", "v"):
+                    assert torch.equal(x[key], y[key]), (l, b, h, key)
+                evicted |= x["n"] < lens[b] + w.decode_steps and x["n_old"] > 0
+    assert evicted and ref.status() == 0 and fused.status() == 0
+    ref.close(); fused.close()
+
+
 def _random_state(rng, n, d, dtype, quantum):
     pos = np.sort(rng.choice(10 * n, size=n, replace=False)).astype(np.int32)
     score = rng.random(n).astype(np.float32)
