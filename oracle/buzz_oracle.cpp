@@ -19,6 +19,14 @@
 //                                (Section 3.3, "BeeHive" and the sentence introducing Alg. 1/2).
 //   * short sequences          : Remark 1 (nothing is evicted while n <= k + w).
 //   * over-long prompts        : Remark 2 (sample repeatedly until the cache fits T + k + w).
+//   * global top-k policy      : the heavy-hitter selection the paper compares against (Section 3.2:
+//                                "top-k tokens based on attention scores A outside the sliding window";
+//                                Section 4.3: a top-k module on accumulated scores "instead of the
+//                                sampling module"). Read here as: at an eviction, sink and window
+//                                stay, and of ALL middle tokens (old and new alike) the M with the
+//                                largest accumulated score survive, M being the number the sampling
+//                                module would have kept, so that both policies run on the same cache
+//                                schedule. Ties go to the lowest position.
 //   * log-n scaled attention   : Section 3.5 (logits scaled by log_512(n)/sqrt(d), n = tokens seen so
 //                                far: row index + 1 at prefill, total length incl. the new token at
 //                                decode -- not the number of retained slots).
@@ -50,6 +58,7 @@ struct Head {
   int logn;            // 0: scale 1/sqrt(d) (Eq. 3); 1: scale log_512(n)/sqrt(d) (Section 3.5)
   int old_stride = 0;  // stride for old tokens; 0 = the paper's s_hat = floor((s+1)/2)
   int interval_new = 0;  // 1: interval sampling for new tokens too (the "no local max" ablation, Section 4.3)
+  int global_topk = 0;   // 1: global top-k of the accumulated scores instead of the sampling module (Sections 3.2, 4.3)
   int n = 0, n_old = 0, total_len = 0;
   std::vector<double> K, V;   // [n][d], position order
   std::vector<double> score;  // [n]
@@ -73,29 +82,20 @@ void softmax_inplace(double* x, int len) {
   for (int j = 0; j < len; ++j) x[j] /= sum;
 }
 
-// One eviction (Algorithm 1, the sampling line and the final concatenation; Algorithm 2).
-// Returns 1 if the cache was rewritten, 0 if the trigger did not fire, <0 on error.
-int evict_once(Head& h) {
-  const int k = h.sink, w = h.window, s = h.segment;
-  if (h.n < h.budget) return 0;          // threshold buffering: evict only when full
-  if (h.n <= k + w) return 0;            // Remark 1: sink and window are filled first
-  const int s_hat = h.old_stride > 0 ? h.old_stride : (s + 1) / 2;   // floor((s+1)/2) unless overridden (Section 4.3)
-  const int new_begin = k + h.n_old;
-  const int new_end = h.n - w;
-
-  std::vector<int> keep;
-  for (int j = 0; j < k; ++j) keep.push_back(j);                       // K[:k]
+// The sampling module (Algorithm 1's sampling line; Algorithm 2): appends to `keep` the surviving
+// middle slots, old region [k, k + n_old) first, then the new region [k + n_old, new_end).
+void sample_middle(const Head& h, int s_hat, int new_end, std::vector<int>& keep) {
+  const int k = h.sink, s = h.segment;
   for (int off = 0; off < h.n_old; off += s_hat) keep.push_back(k + off);  // interval_sample(s_hat, old)
-  int kept_old = (int)keep.size() - k;
   // local_max_sample(s, new): one hive per s consecutive new tokens
-  for (int idx = new_begin; idx < new_end; idx += s) {
+  for (int idx = k + h.n_old; idx < new_end; idx += s) {
     const int hi = std::min(idx + s, new_end);
     const int want = std::min(h.hitters, hi - idx);
-    std::vector<int> chosen;
     if (h.interval_new) {                 // ablation: the first `want` slots of the hive, scores ignored
       for (int r = 0; r < want; ++r) keep.push_back(idx + r);
       continue;
     }
+    std::vector<int> chosen;
     for (int r = 0; r < want; ++r) {
       int best = -1;
       for (int j = idx; j < hi; ++j) {
@@ -107,9 +107,44 @@ int evict_once(Head& h) {
     std::sort(chosen.begin(), chosen.end());
     for (int j : chosen) keep.push_back(j);
   }
+}
+
+// The global top-k module (Sections 3.2 and 4.3): of all middle slots [k, new_end) the M with the
+// largest accumulated score survive, M = the number sample_middle would keep.
+void topk_middle(const Head& h, int s_hat, int new_end, std::vector<int>& keep) {
+  const int k = h.sink, s = h.segment;
+  int M = 0;
+  for (int off = 0; off < h.n_old; off += s_hat) ++M;
+  for (int idx = k + h.n_old; idx < new_end; idx += s) M += std::min(h.hitters, std::min(idx + s, new_end) - idx);
+  // greedy heavy hitters: M times, take the best remaining middle token (first occurrence wins ties)
+  std::vector<int> chosen;
+  for (int r = 0; r < M; ++r) {
+    int best = -1;
+    for (int j = k; j < new_end; ++j) {
+      if (std::find(chosen.begin(), chosen.end(), j) != chosen.end()) continue;
+      if (best < 0 || h.score[j] > h.score[best]) best = j;
+    }
+    chosen.push_back(best);
+  }
+  std::sort(chosen.begin(), chosen.end());
+  for (int j : chosen) keep.push_back(j);
+}
+
+// One eviction (Algorithm 1, the sampling line and the final concatenation; Algorithm 2).
+// Returns 1 if the cache was rewritten, 0 if the trigger did not fire, <0 on error.
+int evict_once(Head& h) {
+  const int k = h.sink, w = h.window, s = h.segment;
+  if (h.n < h.budget) return 0;          // threshold buffering: evict only when full
+  if (h.n <= k + w) return 0;            // Remark 1: sink and window are filled first
+  const int s_hat = h.old_stride > 0 ? h.old_stride : (s + 1) / 2;   // floor((s+1)/2) unless overridden (Section 4.3)
+  const int new_end = h.n - w;
+
+  std::vector<int> keep;
+  for (int j = 0; j < k; ++j) keep.push_back(j);                       // K[:k]
+  if (h.global_topk) topk_middle(h, s_hat, new_end, keep);
+  else sample_middle(h, s_hat, new_end, keep);
   int kept_mid = (int)keep.size() - k;
   for (int j = new_end; j < h.n; ++j) keep.push_back(j);                // K[-w:]
-  (void)kept_old;
 
   const int n2 = (int)keep.size();
   const bool progress = n2 < h.n;
@@ -154,6 +189,14 @@ int bo_set_sampling(void* p, int interval_new, int new_stride, int old_stride) {
   h.segment = new_stride;
   h.old_stride = old_stride;
   h.interval_new = interval_new ? 1 : 0;
+  return BO_OK;
+}
+
+// Selects the eviction policy: 0 = BUZZ's sampling module (Algorithms 1 and 2), 1 = global top-k of
+// the accumulated scores over the whole middle region (the heavy-hitter baseline, Sections 3.2, 4.3).
+int bo_set_policy(void* p, int policy) {
+  if (policy != 0 && policy != 1) return BO_BAD_ARG;
+  ((Head*)p)->global_topk = policy;
   return BO_OK;
 }
 

@@ -55,6 +55,8 @@ def _load():
         lib.bo_set_scores.argtypes = [ctypes.c_void_p, dp]
         lib.bo_set_sampling.restype = c_int
         lib.bo_set_sampling.argtypes = [ctypes.c_void_p, c_int, c_int, c_int]
+        lib.bo_set_policy.restype = c_int
+        lib.bo_set_policy.argtypes = [ctypes.c_void_p, c_int]
         lib.bo_set_state.restype = c_int
         lib.bo_set_state.argtypes = [ctypes.c_void_p, c_int, c_int, c_int, ip, dp, dp, dp]
         _lib = lib
@@ -94,6 +96,11 @@ class OracleHead:
         if rc < 0:
             raise ValueError("oracle rejected the sampling parameters")
         self.segment = int(new_stride)
+
+    def set_policy(self, global_topk):
+        """False: BUZZ's sampling module; True: global top-k of the accumulated scores (Sections 3.2, 4.3)."""
+        if self._lib.bo_set_policy(self._h, int(bool(global_topk))) < 0:
+            raise ValueError("oracle rejected the policy")
 
     # -- the three steps -------------------------------------------------------------------
     def prefill(self, Q, K, V):

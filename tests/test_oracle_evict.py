@@ -300,3 +300,88 @@ def test_sampling_variant_validation():
     for bad in [(False, 1, 2), (False, 3, 2), (False, 8, 0), (False, 40, 2)]:
         with pytest.raises(ValueError):
             h.set_sampling(*bad)
+
+
+# ---- global top-k policy (the heavy-hitter baseline, Sections 3.2 and 4.3) ----------------------
+
+def test_topk_policy_handworked_case():
+    with open(os.path.join(GOLD, "handworked_topk.json")) as f:
+        gold = json.load(f)
+    h = OracleHead(1, 2, **gold["params"])
+    h.set_policy(True)
+    a = gold["first"]
+    _load_state(h, a["pos"], a["score"], a["n_old"])
+    assert h.evict() == 1
+    pos, score, K, V = h.state()
+    assert pos.tolist() == a["expect_pos"] and h.counts()[:2] == (len(a["expect_pos"]), a["expect_n_old"])
+    assert K[:, 0].tolist() == a["expect_pos"]
+    assert score.tolist() == [a["score"][a["pos"].index(p)] for p in a["expect_pos"]]
+    b = gold["second"]
+    pos2 = a["expect_pos"] + b["append_pos"]
+    _load_state(h, pos2, b["score"], a["expect_n_old"])
+    assert h.evict() == 1
+    assert h.state(with_kv=False)[0].tolist() == b["expect_pos"]
+    assert h.counts()[:2] == (len(b["expect_pos"]), b["expect_n_old"])
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_topk_policy_against_a_sort_and_same_schedule_as_sampling(seed):
+    """Random runs with forced ties: the survivors equal a selection written independently here (sort
+    the middle slots by (score descending, slot ascending), cut at M, restore slot order), M follows
+    the sampling module's count rule, and so the (n, n_old) trajectory is the one the sampling
+    policy produces on the same lengths."""
+    rng = np.random.default_rng(100 + seed)
+    sink = int(rng.integers(0, 5)); window = int(rng.integers(1, 20)); s = int(rng.integers(3, 12))
+    hit = int(rng.integers(1, min(s, 4))); budget = sink + window + s + int(rng.integers(0, 120))
+    top, ref = OracleHead(1, 1, sink, window, s, hit, budget), OracleHead(1, 1, sink, window, s, hit, budget)
+    top.set_policy(True)
+    z = np.zeros((1, 1))
+    for head in (top, ref):
+        head.prefill(z[None], z, z)
+    s_hat = (s + 1) // 2
+    evictions = 0
+    for t in range(1, 500):
+        for head in (top, ref):
+            head.decode(z, z[0], z[0])
+        n, n_old, tot = top.counts()
+        assert ref.counts() == (n, n_old, tot)                       # same schedule under both policies
+        sc = np.round(rng.random(n) * 6) / 6                         # many exact ties
+        top.set_scores(sc); ref.set_scores(sc)
+        pos, _ = top.state(with_kv=False)
+        r = top.evict()
+        assert ref.evict() == r
+        if n < budget:
+            assert r == 0
+            continue
+        assert r == 1
+        evictions += 1
+        lo, hi = sink, n - window
+        M = len(range(0, n_old, s_hat)) + sum(min(hit, min(a + s, hi) - a) for a in range(sink + n_old, hi, s))
+        chosen = sorted(sorted(range(lo, hi), key=lambda j: (-sc[j], j))[:M])
+        expect = list(range(sink)) + chosen + list(range(hi, n))
+        pos2, sc2 = top.state(with_kv=False)
+        assert pos2.tolist() == pos[expect].tolist()
+        np.testing.assert_array_equal(sc2, sc[expect])
+        assert top.counts()[1] == M
+        assert np.all(np.diff(pos2) > 0) and pos2[-window:].tolist() == list(range(t + 1 - window, t + 1))
+        # every survivor's score is >= every evicted middle token's score
+        evicted = sorted(set(range(lo, hi)) - set(chosen))
+        if evicted and chosen:
+            assert min(sc[j] for j in chosen) >= max(sc[j] for j in evicted)
+    assert evictions >= 3
+
+
+def test_topk_policy_at_prefill_keeps_the_overall_heaviest():
+    """Remark 2's repeated rounds under the top-k policy: top-k sets are nested, so after any number
+    of rounds the middle survivors are the M_final heaviest prompt tokens between sink and window."""
+    sink, window, s, budget, N, d = 4, 32, 8, 100, 1500, 2
+    rng = np.random.default_rng(9)
+    Q, K, V = rng.standard_normal((1, N, d)), rng.standard_normal((N, d)), rng.standard_normal((N, d))
+    h = OracleHead(1, d, sink, window, s, 1, budget)
+    h.set_policy(True)
+    _, full, rounds = h.prefill(Q, K, V)
+    assert rounds >= 2
+    M = h.counts()[1]
+    mid = range(sink, N - window)
+    chosen = sorted(sorted(mid, key=lambda j: (-full[j], j))[:M])
+    assert h.state(with_kv=False)[0].tolist() == list(range(sink)) + chosen + list(range(N - window, N))
