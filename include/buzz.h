@@ -63,6 +63,11 @@ enum {
   BUZZ_FLAG_LOGN = 1         /* scale logits by log_512(tokens seen)/sqrt(d) (Section 3.5)   */
 };
 
+enum {
+  BUZZ_POLICY_BEEHIVE = 0,     /* BUZZ's sampling module: Algorithms 1 and 2 (the default)        */
+  BUZZ_POLICY_GLOBAL_TOPK = 1  /* global top-k of the accumulated scores (Sections 3.2 and 4.3)   */
+};
+
 /* Sizes of the two device allocations buzz_create needs (Section 3.3 fixes the cache at
  * budget = T + sink + window slots per instance).
  *   state   : K and V caches [L][max_batch][Hkv][budget][d], score and pos [L][max_batch][Hkv][budget],
@@ -248,6 +253,16 @@ int64_t buzz_launch_count(buzz_t ctx);
  * scores are ignored). Takes effect from the next prefill / eviction; counts stay score-independent.
  * Rejects new_stride < 2, hitters >= new_stride, old_stride < 1, budget < sink + window + new_stride. */
 int buzz_set_sampling(buzz_t ctx, int interval_new, int new_stride, int old_stride);
+
+/* Eviction policy. BUZZ_POLICY_BEEHIVE is the paper's method. BUZZ_POLICY_GLOBAL_TOPK is the
+ * heavy-hitter selection the paper compares against (Section 3.2, "top-k tokens based on attention
+ * scores A outside the sliding window"; Section 4.3, a top-k module on accumulated scores "instead of
+ * the sampling module"): sink and window are kept as always, and of ALL tokens in between, old and
+ * new alike, the M with the largest accumulated score survive (ties to the lowest position, emitted
+ * in position order), where M is the number of tokens the sampling module would have kept at that
+ * eviction, so that both policies follow the same cache-length schedule. Applies to prefill-time
+ * rounds and decode-time evictions from the next call on. Rejects an unknown policy. */
+int buzz_set_policy(buzz_t ctx, int policy);
 
 /* Tuning knob: number of CTAs (1, 2, 4 or 8) of the thread-block cluster that shares one instance's
  * slots in buzz_decode_step; 0 restores the built-in choice. Results do not depend on it beyond

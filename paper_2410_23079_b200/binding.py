@@ -38,7 +38,7 @@ def exported_symbols() -> list[str]:
             "buzz_decode_step_host", "buzz_decode_layers", "buzz_decode_layers_host", "buzz_evict", "buzz_export_state", "buzz_import_state",
             "buzz_export_prefill_scores", "buzz_prefill_static", "buzz_selftest_wait_expiry",
             "buzz_status", "buzz_launch_count", "buzz_set_decode_cluster", "buzz_set_sampling", "buzz_set_fused_evict",
-            "buzz_error_string"]
+            "buzz_set_policy", "buzz_error_string"]
 
 
 def load_library(build_if_missing: bool = True):
@@ -87,6 +87,8 @@ def load_library(build_if_missing: bool = True):
     lib.buzz_launch_count.argtypes = [vp]
     lib.buzz_set_sampling.restype = ci
     lib.buzz_set_sampling.argtypes = [vp, ci, ci, ci]
+    lib.buzz_set_policy.restype = ci
+    lib.buzz_set_policy.argtypes = [vp, ci]
     lib.buzz_set_fused_evict.restype = ci
     lib.buzz_set_fused_evict.argtypes = [vp, ci]
     lib.buzz_set_decode_cluster.restype = ci
@@ -214,6 +216,10 @@ class Buzz:
 
     def set_sampling(self, interval_new: bool, new_stride: int, old_stride: int):
         _check(self._lib.buzz_set_sampling(self._h, int(bool(interval_new)), new_stride, old_stride), "buzz_set_sampling")
+
+    def set_policy(self, global_topk: bool):
+        """buzz_set_policy: False = BUZZ's sampling module, True = global top-k of the accumulated scores."""
+        _check(self._lib.buzz_set_policy(self._h, 1 if global_topk else 0), "buzz_set_policy")
 
     def set_fused_evict(self, on: bool):
         """buzz_set_fused_evict: decode steps run the eviction of a cache they fill in their own tail."""

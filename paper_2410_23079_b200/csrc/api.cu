@@ -113,7 +113,7 @@ int buzz_create(buzz_t* out, int sink, int window, int segment, int hitters, int
     return BUZZ_ERR_INVALID;
   buzz_ctx* c = new (std::nothrow) buzz_ctx();
   if (!c) return BUZZ_ERR_INVALID;
-  c->pol = BuzzPolicy{sink, window, segment, hitters, budget, (segment + 1) / 2, 0};
+  c->pol = BuzzPolicy{sink, window, segment, hitters, budget, (segment + 1) / 2, 0, BUZZ_POLICY_BEEHIVE};
   c->sh = *shape;
   c->group = shape->q_heads / shape->kv_heads;
   c->esize = shape->dtype == BUZZ_BF16 ? 2 : 4;
@@ -452,6 +452,12 @@ int buzz_set_sampling(buzz_t c, int interval_new, int new_stride, int old_stride
   c->pol.segment = new_stride;
   c->pol.s_hat = old_stride;
   c->pol.interval_new = interval_new ? 1 : 0;
+  return BUZZ_OK;
+}
+
+int buzz_set_policy(buzz_t c, int policy) {
+  if (!c || (policy != BUZZ_POLICY_BEEHIVE && policy != BUZZ_POLICY_GLOBAL_TOPK)) return BUZZ_ERR_INVALID;
+  c->pol.policy = policy;
   return BUZZ_OK;
 }
 

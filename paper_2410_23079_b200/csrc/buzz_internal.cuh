@@ -17,6 +17,7 @@ struct BuzzPolicy {
   int budget;    // T + k + w
   int s_hat;     // stride for old tokens: floor((s+1)/2) unless overridden
   int interval_new;  // 1: interval sampling for new tokens too (ablation), 0: local max (Algorithm 2)
+  int policy;        // BUZZ_POLICY_BEEHIVE (sampling module) or BUZZ_POLICY_GLOBAL_TOPK
 };
 
 // Device view of the persistent state. Instance index = ((layer * max_batch) + seq) * kv_heads + head.

@@ -72,6 +72,108 @@ __device__ inline Cand better(Cand a, Cand b) {
   return a;
 }
 
+// Order-preserving key of a score: a larger float gives a larger unsigned integer (-0 counts as +0).
+__device__ inline uint32_t order_key(float v) {
+  const uint32_t b = __float_as_uint(v + 0.0f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+// Global top-M selection by one whole CTA (the heavy-hitter policy the paper compares against,
+// Sections 3.2 and 4.3): of cand[0 .. count) the M largest survive, equal scores going to the lowest
+// index; emit(t, j) is called once per survivor, t = its rank in index order, j = its index.
+// Exact and deterministic: a four-pass radix select (8 bits per pass, shared-memory histogram with
+// warp-aggregated increments) finds the M-th largest key and how many keys equal to it survive; one
+// ordered pass over the candidates then hands out the ranks with ballots and popcounts.
+template <int THREADS, typename Emit>
+__device__ void topk_select(const float* __restrict__ cand, int count, int M, Emit emit) {
+  __shared__ int hist[256];
+  __shared__ int warp_cnt[2][THREADS / 32];
+  __shared__ uint32_t found_prefix;
+  __shared__ int found_remaining;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (M <= 0) return;
+  if (M >= count) {
+    for (int j = tid; j < count; j += THREADS) emit(j, j);
+    return;
+  }
+  uint32_t prefix = 0, mask = 0;
+  int remaining = M;                       // survivors still to be found among the keys matching `prefix`
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    for (int i = tid; i < 256; i += THREADS) hist[i] = 0;
+    __syncthreads();
+    for (int base = 0; base < count; base += THREADS) {
+      const int j = base + tid;
+      int bin = -1;
+      if (j < count) {
+        const uint32_t key = order_key(cand[j]);
+        if ((key & mask) == prefix) bin = (int)((key >> shift) & 255u);
+      }
+      const unsigned peers = __match_any_sync(0xffffffffu, bin);
+      if (bin >= 0 && lane == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
+    }
+    __syncthreads();
+    if (warp == 0) {                       // lane l owns bins 8l .. 8l+7; walk from the top bin down
+      int c[8], mine = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { c[i] = hist[8 * lane + i]; mine += c[i]; }
+      int incl = mine;                     // keys in this lane's bins and all higher lanes' bins
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int o = __shfl_down_sync(0xffffffffu, incl, off);
+        if (lane + off < 32) incl += o;
+      }
+      int cum = incl - mine;               // keys in strictly higher bins than this lane's
+#pragma unroll
+      for (int i = 7; i >= 0; --i) {
+        if (cum < remaining && cum + c[i] >= remaining) {
+          found_prefix = prefix | ((uint32_t)(8 * lane + i) << shift);
+          found_remaining = remaining - cum;
+        }
+        cum += c[i];
+      }
+    }
+    __syncthreads();
+    prefix = found_prefix;
+    remaining = found_remaining;
+    mask |= 255u << shift;
+  }
+  // prefix is now the M-th largest key; `remaining` of the keys equal to it survive, lowest index first
+  int eq_base = 0, out_base = 0;
+  for (int base = 0; base < count; base += THREADS) {
+    const int j = base + tid;
+    bool gt = false, eq = false;
+    if (j < count) {
+      const uint32_t key = order_key(cand[j]);
+      gt = key > prefix;
+      eq = key == prefix;
+    }
+    const unsigned lower = (1u << lane) - 1u;
+    const unsigned be = __ballot_sync(0xffffffffu, eq);
+    if (lane == 0) warp_cnt[0][warp] = __popc(be);
+    __syncthreads();
+    int eq_before = eq_base + __popc(be & lower), eq_total = 0;
+#pragma unroll
+    for (int w = 0; w < THREADS / 32; ++w) {
+      if (w < warp) eq_before += warp_cnt[0][w];
+      eq_total += warp_cnt[0][w];
+    }
+    const bool take = gt || (eq && eq_before < remaining);
+    const unsigned bt = __ballot_sync(0xffffffffu, take);
+    if (lane == 0) warp_cnt[1][warp] = __popc(bt);
+    __syncthreads();
+    int out = out_base + __popc(bt & lower), take_total = 0;
+#pragma unroll
+    for (int w = 0; w < THREADS / 32; ++w) {
+      if (w < warp) out += warp_cnt[1][w];
+      take_total += warp_cnt[1][w];
+    }
+    if (take) emit(out, j);
+    eq_base += eq_total;
+    out_base += take_total;
+  }
+}
+
 // One eviction of one instance by one whole CTA of THREADS threads (all of them must call it; the
 // trigger n >= budget and Remark 1's n > sink + window are the caller's to check).
 //   old region  [mb, mb + n_old)   keep offsets 0, s_hat, 2 s_hat, ...          (interval sampling)
@@ -80,8 +182,10 @@ __device__ inline Cand better(Cand a, Cand b) {
 // with mb = sink + window. The counts depend only on n and n_old, so every destination is closed-form;
 // only the winners inside a segment depend on the scores. A warp owns a segment: each lane holds the
 // candidates lane, lane+32, ...; h rounds of a shuffle arg-max flag the winners, ballots + popcounts
-// give their rank in position order. Compaction is an in-place stable left shift (destination <=
-// source): ascending chunks, a chunk's sources read into registers, a barrier, then the writes.
+// give their rank in position order. Under the global top-k policy the same number of survivors is
+// taken from the whole middle region by score alone (topk_select). Compaction is an in-place stable
+// left shift (destination <= source): ascending chunks, a chunk's sources read into registers, a
+// barrier, then the writes.
 // `src` is shared memory for at least kept_old + kept_new ints (never more than n - sink - window).
 template <int ROW_BYTES, int THREADS>
 __device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_t inst, int n, int n_old,
@@ -102,39 +206,43 @@ __device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_
   int32_t* pos = st.pos + inst * pol.budget;
 
   // ---- selection: src[t] = source slot of middle destination mb + t ---------------------------
-  for (int t = tid; t < kept_old; t += THREADS) src[t] = mb + t * s_hat;
-  for (int seg = warp; seg < nseg; seg += THREADS / 32) {
-    const int lo = new_begin + seg * s;
-    const int len = min(s, n - lo);
-    const int want = min(h, len);
-    const int out0 = kept_old + seg * h;
-    if (pol.interval_new) {                         // ablation: the first `want` slots of the segment
-      for (int r = lane; r < want; r += 32) src[out0 + r] = lo + r;
-      continue;
-    }
-    unsigned chosen = 0;                            // bit i: candidate lo + i*32 + lane is a winner
-    for (int r = 0; r < want; ++r) {
-      Cand best{0.f, -1};
-      for (int i = 0, j = lane; j < len; ++i, j += 32) {
-        if (chosen >> i & 1u) continue;
-        best = better(best, Cand{score[lo + j], lo + j});
+  if (pol.policy == BUZZ_POLICY_GLOBAL_TOPK) {
+    topk_select<THREADS>(score + mb, n - mb, kept_mid, [&](int t, int j) { src[t] = mb + j; });
+  } else {
+    for (int t = tid; t < kept_old; t += THREADS) src[t] = mb + t * s_hat;
+    for (int seg = warp; seg < nseg; seg += THREADS / 32) {
+      const int lo = new_begin + seg * s;
+      const int len = min(s, n - lo);
+      const int want = min(h, len);
+      const int out0 = kept_old + seg * h;
+      if (pol.interval_new) {                         // ablation: the first `want` slots of the segment
+        for (int r = lane; r < want; r += 32) src[out0 + r] = lo + r;
+        continue;
       }
+      unsigned chosen = 0;                            // bit i: candidate lo + i*32 + lane is a winner
+      for (int r = 0; r < want; ++r) {
+        Cand best{0.f, -1};
+        for (int i = 0, j = lane; j < len; ++i, j += 32) {
+          if (chosen >> i & 1u) continue;
+          best = better(best, Cand{score[lo + j], lo + j});
+        }
 #pragma unroll
-      for (int off = 16; off > 0; off >>= 1) {
-        Cand o;
-        o.v = __shfl_xor_sync(0xffffffffu, best.v, off);
-        o.idx = __shfl_xor_sync(0xffffffffu, best.idx, off);
-        best = better(best, o);
+        for (int off = 16; off > 0; off >>= 1) {
+          Cand o;
+          o.v = __shfl_xor_sync(0xffffffffu, best.v, off);
+          o.idx = __shfl_xor_sync(0xffffffffu, best.idx, off);
+          best = better(best, o);
+        }
+        const int w = best.idx - lo;
+        if ((w & 31) == lane) chosen |= 1u << (w >> 5);
       }
-      const int w = best.idx - lo;
-      if ((w & 31) == lane) chosen |= 1u << (w >> 5);
-    }
-    int before = 0;                                 // winners at lower positions
-    for (int i = 0; i * 32 < len; ++i) {
-      const bool mine = chosen >> i & 1u;
-      const unsigned b = __ballot_sync(0xffffffffu, mine);
-      if (mine) src[out0 + before + __popc(b & ((1u << lane) - 1u))] = lo + i * 32 + lane;
-      before += __popc(b);
+      int before = 0;                                 // winners at lower positions
+      for (int i = 0; i * 32 < len; ++i) {
+        const bool mine = chosen >> i & 1u;
+        const unsigned b = __ballot_sync(0xffffffffu, mine);
+        if (mine) src[out0 + before + __popc(b & ((1u << lane) - 1u))] = lo + i * 32 + lane;
+        before += __popc(b);
+      }
     }
   }
   __syncthreads();
@@ -155,8 +263,8 @@ __device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_
   uint4* Kc = reinterpret_cast<uint4*>(st.K + inst * (size_t)pol.budget * ROW_BYTES);
   uint4* Vc = reinterpret_cast<uint4*>(st.V + inst * (size_t)pol.budget * ROW_BYTES);
   const int sub = tid % LPR, rgrp = tid / LPR;
-  // The first old survivor stays where it is.
-  for (int base = kept_old > 0 ? 1 : 0; base < kept_mid; base += ROWS) {
+  // Under the sampling policy the first old survivor stays where it is.
+  for (int base = (kept_old > 0 && pol.policy != BUZZ_POLICY_GLOBAL_TOPK) ? 1 : 0; base < kept_mid; base += ROWS) {
     uint4 kr[kRowsPerPass], vr[kRowsPerPass];
 #pragma unroll
     for (int u = 0; u < kRowsPerPass; ++u) {

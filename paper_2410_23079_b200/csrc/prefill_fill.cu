@@ -10,7 +10,11 @@
 // one segment of <= s scores) and copies that row. The cache is laid out [sink | window ring |
 // middle] (cache_ops.cuh): the prompt's last `window` tokens fill the ring in order (head 0) and
 // the survivors between sink and window follow it.
-#include "buzz_internal.cuh"
+// Under the global top-k policy the rounds are nested (the heaviest M2 of the heaviest M1 are the
+// heaviest M2), so the middle survivors are simply the n_mid heaviest prompt tokens between sink
+// and window: one CTA per instance selects them first and leaves their token indices in the cache's
+// position array, where the gather then finds its sources.
+#include "cache_ops.cuh"
 
 namespace {
 
@@ -77,6 +81,20 @@ __device__ inline int round_one_winner(const float* __restrict__ sc, int N, cons
   return lo;   // unreachable for NaN-free scores
 }
 
+// Global top-k policy: the middle survivors of one instance, in position order, into pos[middle slots].
+__global__ void __launch_bounds__(kThreads)
+prefill_topk_kernel(BuzzState st, BuzzPolicy pol, const int32_t* __restrict__ cu, const float* __restrict__ pscore,
+                    int stride, int layer, int max_batch, int kv_heads) {
+  const int head = blockIdx.x, seq = blockIdx.y;
+  const size_t inst = ((size_t)layer * max_batch + seq) * kv_heads + head;
+  const int tok0 = cu[seq], N = cu[seq + 1] - tok0;
+  const FillPlan plan = make_plan(N, pol);
+  if (plan.error || plan.rounds == 0) return;
+  int32_t* mid_pos = st.pos + inst * (size_t)pol.budget + buzz_dev::middle_begin(pol);
+  buzz_dev::topk_select<kThreads>(pscore + (size_t)head * stride + tok0 + pol.sink, N - pol.sink - pol.window,
+                                  plan.n_mid, [&](int t, int j) { mid_pos[t] = pol.sink + j; });
+}
+
 template <int ROW_BYTES>
 __global__ void __launch_bounds__(kThreads)
 prefill_fill_kernel(BuzzState st, BuzzPolicy pol, const char* __restrict__ k, const char* __restrict__ v,
@@ -106,7 +124,9 @@ prefill_fill_kernel(BuzzState st, BuzzPolicy pol, const char* __restrict__ k, co
   for (int t = blockIdx.x * SLOTS + grp; t < plan.n_final; t += gridDim.x * SLOTS) {
     int src;
     if (plan.rounds == 0 || t < pol.sink) src = t;
-    else if (t < pol.sink + plan.n_mid) src = round_one_winner(sc, N, pol, (int)((t - pol.sink) * plan.stride));
+    else if (t < pol.sink + plan.n_mid)
+      src = pol.policy == BUZZ_POLICY_GLOBAL_TOPK ? st.pos[cache_row0 + t + pol.window]   // left there by prefill_topk_kernel
+                                                  : round_one_winner(sc, N, pol, (int)((t - pol.sink) * plan.stride));
     else src = N - pol.window + (t - pol.sink - plan.n_mid);
     // t counts the survivors in position order; their slots: sink, then (behind the ring) the middle,
     // and the last `window` tokens in the ring right after the sink
@@ -135,6 +155,12 @@ cudaError_t buzz_launch_prefill_fill(buzz_ctx* c, int layer, const void* k, cons
   if (bx < 1) bx = 1;
   dim3 grid(bx, c->sh.kv_heads, batch);
   (void)cudaGetLastError();   // drop a stale non-sticky error left by an earlier runtime call of the process
+  if (c->pol.policy == BUZZ_POLICY_GLOBAL_TOPK) {
+    prefill_topk_kernel<<<dim3(c->sh.kv_heads, batch), kThreads, 0, stream>>>(
+        c->st, c->pol, cu, c->pscore, c->sh.max_prompt_tokens, layer, c->sh.max_batch, c->sh.kv_heads);
+    c->launches += 1;
+    if (cudaError_t e = cudaGetLastError(); e != cudaSuccess) return e;
+  }
 #define BUZZ_FILL_CASE(RB)                                                                      \
   case RB:                                                                                      \
     prefill_fill_kernel<RB><<<grid, kThreads, 0, stream>>>(                                     \

@@ -82,7 +82,8 @@ def check_free_running(fr: OracleHead, before, gpu_pos, w, what, stats):
         a, b = score_of[pf], score_of[pg]
         assert abs(a - b) <= SCORE_RTOL * max(abs(a), abs(b)), \
             f"{what}: GPU kept position {pg} (score {b}) where the oracle kept {pf} (score {a}): not a near-tie"
-        assert abs(slot_of[pf] - slot_of[pg]) < fr.segment, f"{what}: positions {pf}, {pg} are not in one segment"
+        if not getattr(fr, "global_topk", False):           # the sampling module decides inside one segment
+            assert abs(slot_of[pf] - slot_of[pg]) < fr.segment, f"{what}: positions {pf}, {pg} are not in one segment"
     stats["free_running_evictions"] += 1
     stats["free_running_near_ties"] += len(only_f)
     return len(only_f) == 0
@@ -117,7 +118,7 @@ def check_prefill_sampled(w, Q, K, V, got, gpu_scores, rows, tail_keys, tol, log
 
 def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None, check_every=1,
                  device="cuda:0", logn=False, bz: Buzz | None = None, sampled_rows=None, tail_keys=64,
-                 sampling=None, layers_call=False):
+                 sampling=None, layers_call=False, topk=False):
     """Runs prefill + decode/evict on the GPU for the whole workload and the oracle on `samples`
     (a list of (layer, seq, kv_head)). Returns a dict of summary counters."""
     tol = TOL[w.dtype]
@@ -127,6 +128,18 @@ def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None,
     bz = bz or make_buzz(w, device, logn=logn)
     if sampling is not None:                     # (interval_new, new_stride, old_stride): Section 4.3 variants
         bz.set_sampling(*sampling)
+    if topk:                                     # global top-k policy instead of the sampling module
+        bz.set_policy(True)
+
+    def new_oracle(budget=w.budget):
+        o = OracleHead(g, d, w.sink, w.window, w.segment, w.hitters, budget, logn=logn)
+        if sampling is not None:
+            o.set_sampling(*sampling)
+        if topk:
+            o.set_policy(True)
+            o.global_topk = True
+        return o
+
     lens = workloads.prompt_lengths(w)
     offs = np.concatenate([[0], np.cumsum(lens)])
     g, d = w.group, w.head_dim
@@ -152,9 +165,7 @@ def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None,
                 pscore[h] = bz.export_prefill_scores(h, int(offs[-1])).numpy()
             gs = pscore[h][a:e]
             if sampled_rows is None:
-                free = OracleHead(g, d, w.sink, w.window, w.segment, w.hitters, w.budget, logn=logn)
-                if sampling is not None:
-                    free.set_sampling(*sampling)
+                free = new_oracle()
                 O, full, rounds = free.prefill(Q, K, V)
                 stats["prefill_rounds"] = max(stats["prefill_rounds"], rounds)
                 assert_close(got, O, what=f"prefill out L{layer} b{b} h{h}", **tol)
@@ -165,9 +176,7 @@ def run_lockstep(w: workloads.Workload, samples, decode_steps=None, layers=None,
                 check_prefill_sampled(w, Q, K, V, got, gs, sampled_rows, tail_keys, tol, logn,
                                       f"L{layer} b{b} h{h}", stats)
             # lock-step instance: selection decided on the GPU's fp32 scores
-            ls = OracleHead(g, d, w.sink, w.window, w.segment, w.hitters, w.budget, logn=logn)
-            if sampling is not None:
-                ls.set_sampling(*sampling)
+            ls = new_oracle()
             N = e - a
             ls.set_state(0, N, np.arange(N), gs.astype(np.float64), K, V)
             while ls.counts()[0] >= w.budget:
