@@ -60,6 +60,25 @@ __device__ inline void append_rows(const BuzzState& st, const BuzzPolicy& pol, s
   }
 }
 
+// The same stores from rows staged in shared memory by the calling threads themselves: stage[0, LPR)
+// and [LPR, 2 LPR) hold the K and V rows of the token that leaves the window (if any), the next 2 LPR
+// entries the appended token's K and V rows, *stage_pos the leaving token's position. Thread t reads
+// only what thread t staged, so no barrier is needed between staging and this call.
+template <int LPR>
+__device__ inline void append_staged(const BuzzState& st, const BuzzPolicy& pol, size_t inst, const AppendPlan& a,
+                                     int tot, const uint4* stage, const int32_t* stage_pos, int tid) {
+  int32_t* pos = st.pos + inst * pol.budget;
+  if (tid < 2 * LPR) {
+    uint4* cache = reinterpret_cast<uint4*>(tid < LPR ? st.K : st.V) + inst * (size_t)pol.budget * LPR;
+    const int t = tid < LPR ? tid : tid - LPR;
+    if (a.slot_moved >= 0) cache[(size_t)a.slot_moved * LPR + t] = stage[tid];
+    cache[(size_t)a.slot_new * LPR + t] = stage[2 * LPR + tid];
+  } else if (tid == 2 * LPR) {
+    if (a.slot_moved >= 0) pos[a.slot_moved] = *stage_pos;
+    pos[a.slot_new] = tot;
+  }
+}
+
 struct Cand {
   float v;
   int idx;   // slot index, -1 = none

@@ -43,6 +43,16 @@ constexpr int kAhead = 2;   // rolling L2 prefetch runs this many loop iteration
 
 __device__ inline uint4 ld_stream(const uint4* p) { return __ldcs(p); }
 
+// Asynchronous global -> shared copies (no register, no stall at issue); a thread that later reads
+// what it copied itself only needs its own cp_async_wait().
+__device__ inline void cp_async16(void* dst_smem, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_smem)), "l"(src) : "memory");
+}
+__device__ inline void cp_async4(void* dst_smem, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_smem)), "l"(src) : "memory");
+}
+__device__ inline void cp_async_wait() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 __device__ inline void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                 uint32_t b0, uint32_t b1) {
   asm volatile(
@@ -59,6 +69,9 @@ __device__ inline uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&p);
 }
+
+template <int D>
+constexpr int kStageBytes = 4 * (D / 8) * 16 + 16;
 
 template <int G, int D>
 struct Partial {       // what a CTA publishes to its cluster
@@ -87,7 +100,11 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   const int r8 = lane >> 2, c4 = lane & 3;
 
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  Partial<G, D>* part = reinterpret_cast<Partial<G, D>*>(smem_raw);
+  // rows the append will store after the cluster barrier, fetched asynchronously at the start (CTA 0):
+  // [0, NCH) the window token that moves to the middle (K), [NCH, 2 NCH) its V, then the new K and V rows
+  uint4* stage = reinterpret_cast<uint4*>(smem_raw);
+  int32_t* stage_pos = reinterpret_cast<int32_t*>(stage + 4 * NCH);     // position of the moving token
+  Partial<G, D>* part = reinterpret_cast<Partial<G, D>*>(smem_raw + kStageBytes<D>);
   float* red = reinterpret_cast<float*>(part + 1);           // [kWarps][kHeads]
   float* mloc = red + kWarps * kHeads;                       // [kHeads] chunk-local max
   float* fr = mloc + kHeads;                                 // [kMaxCluster][G] merge factors
@@ -147,6 +164,16 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   // stored only after the cluster barrier below, because with a full window ring it replaces the
   // oldest window token, whose row other CTAs are still reading until then.
   const buzz_dev::AppendPlan app = buzz_dev::plan_append(pol, n0, ring_head);
+  if (rank == 0) {   // nobody writes these rows before the barrier, so they can be fetched now and only stored in the tail
+    if (tid < 2 * NCH) {
+      const uint4* cache = tid < NCH ? Kc : Vc;
+      const int t = tid < NCH ? tid : tid - NCH;
+      if (app.slot_moved >= 0) cp_async16(stage + tid, cache + (size_t)app.slot_new * NCH + t);
+      cp_async16(stage + 2 * NCH + tid, (tid < NCH ? knew : vnew) + t);
+    } else if (tid == 2 * NCH && app.slot_moved >= 0) {
+      cp_async4(stage_pos, st.pos + inst * pol.budget + app.slot_new);
+    }
+  }
 
   // Rolling L2 prefetch. The CTA's traffic is one stream: its K rows, then its V rows, then (as a
   // hint only) the head of the same chunk in the NEXT layer's K cache, which the next decode launch
@@ -331,7 +358,8 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   cluster.sync();
   if (mode == kOverlap) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (rank == 0) {                   // every CTA has read n0/tot/ring and all old rows before the barrier
-    buzz_dev::append_rows<NCH>(st, pol, inst, app, tot, knew, vnew, tid);
+    if (tid <= 2 * NCH) cp_async_wait();
+    buzz_dev::append_staged<NCH>(st, pol, inst, app, tot, stage, stage_pos, tid);
     if (tid == kThreads - 1) {
       st.n[inst] = n1;
       st.total[inst] = tot + 1;
@@ -397,7 +425,7 @@ cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, con
                    void* out, int cluster_size, int mode, int next_layer, cudaStream_t stream) {
   const int batch = c->batch[layer];
   const int chunk_cap = (((c->pol.budget + cluster_size - 1) / cluster_size + 1) & ~1) + 2;
-  const size_t smem = sizeof(Partial<G, D>) +
+  const size_t smem = kStageBytes<D> + sizeof(Partial<G, D>) +
                       sizeof(float) * (kWarps * kHeads + kHeads + kMaxCluster * G + 2 * G +
                                        kWarps * G * D + (size_t)G * chunk_cap) +
                       (c->fused_evict ? sizeof(int32_t) * (size_t)(c->pol.budget - c->pol.sink - c->pol.window) : 0);
