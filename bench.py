@@ -194,17 +194,21 @@ def _warm_library(w, dt, dev):
 class Leg:
     """CUDA-event timing of a run of steps on the launching stream."""
 
-    def __init__(self, stream):
-        self.stream = stream
+    def __init__(self, stream, name=None):
+        self.stream, self.name = stream, name              # name: an NVTX range a profiler can filter on
         self.a, self.b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
     def __enter__(self):
         torch.cuda.synchronize()
+        if self.name:
+            torch.cuda.nvtx.range_push(self.name)
         self.a.record(self.stream)
         return self
 
     def __exit__(self, *exc):
         self.b.record(self.stream)
+        if self.name:
+            torch.cuda.nvtx.range_pop()
         torch.cuda.synchronize()
         self.ms = self.a.elapsed_time(self.b)
 
@@ -232,7 +236,7 @@ def measure(w, K, W, peaks, dev, dist, world, *, headline, e2e_steps=0, evict_le
     for layer in range(w.layers):
         q, k, v, cu = workloads.prefill_inputs(w, layer, dev)
         out = torch.empty_like(q)
-        with Leg(stream) as leg:
+        with Leg(stream, "prefill") as leg:
             bz.prefill(layer, q, k, v, cu, max(lens), out)
         pre_ms += leg.ms
         del q, k, v, out
@@ -426,7 +430,7 @@ def measure(w, K, W, peaks, dev, dist, world, *, headline, e2e_steps=0, evict_le
             step_layers()
             timed = due or idle_calls < 8
             if timed:
-                with Leg(stream) as leg:
+                with Leg(stream, "evict_due" if due else None) as leg:
                     bz.evict(-1)
             else:
                 bz.evict(-1)

@@ -193,26 +193,37 @@ __device__ void topk_select(const float* __restrict__ cand, int count, int M, Em
   }
 }
 
+// Shared memory one eviction needs: the source-slot list, and (when it fits) a staged copy of the
+// middle region's scores and positions, so that the selection reads no global memory at all.
+constexpr int kEvictStageLimit = 5440;        // middle-region capacity up to which scores and positions are staged
+__host__ __device__ inline bool evict_staged(const BuzzPolicy& p) { return p.budget - middle_begin(p) <= kEvictStageLimit; }
+__host__ __device__ inline size_t evict_smem_bytes(const BuzzPolicy& p) {
+  return (size_t)(p.budget - middle_begin(p)) * 4u * (evict_staged(p) ? 3u : 1u);
+}
+
 // One eviction of one instance by one whole CTA of THREADS threads (all of them must call it; the
 // trigger n >= budget and Remark 1's n > sink + window are the caller's to check).
 //   old region  [mb, mb + n_old)   keep offsets 0, s_hat, 2 s_hat, ...          (interval sampling)
 //   new region  [mb + n_old, n)    per segment of s slots keep the top-h by (score desc, position asc),
 //                                  in position order                            (Algorithm 2)
 // with mb = sink + window. The counts depend only on n and n_old, so every destination is closed-form;
-// only the winners inside a segment depend on the scores. A warp owns a segment: each lane holds the
-// candidates lane, lane+32, ...; h rounds of a shuffle arg-max flag the winners, ballots + popcounts
-// give their rank in position order. Under the global top-k policy the same number of survivors is
-// taken from the whole middle region by score alone (topk_select). Compaction is an in-place stable
-// left shift (destination <= source): ascending chunks, a chunk's sources read into registers, a
-// barrier, then the writes.
-// `src` is shared memory for at least kept_old + kept_new ints (never more than n - sink - window).
+// only the winners inside a segment depend on the scores. The middle region's scores and positions
+// are first copied to shared memory with coalesced loads (one memory latency instead of one per
+// segment). A warp owns a segment: each lane holds the candidates lane, lane+32, ...; h rounds of a
+// shuffle arg-max flag the winners, ballots + popcounts give their rank in position order. Under the
+// global top-k policy the same number of survivors is taken from the whole middle region by score
+// alone (topk_select). Compaction is an in-place stable left shift (destination <= source):
+// ascending chunks, a chunk's sources read into registers, a barrier, then the writes.
+// `work` is shared memory of evict_smem_bytes(pol) bytes.
 template <int ROW_BYTES, int THREADS>
 __device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_t inst, int n, int n_old,
-                               int32_t* src) {
+                               int32_t* work) {
   constexpr int kRowsPerPass = 4;   // rows of K and of V each 16-byte lane moves per pass
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int s = pol.segment, h = pol.hitters, s_hat = pol.s_hat;
   const int mb = middle_begin(pol);
+  const int cap = pol.budget - mb;                   // capacity of the middle region
+  const int m = n - mb;                              // its occupancy
   const int new_begin = mb + n_old;
   const int n_new = n - new_begin;
   const int kept_old = (n_old + s_hat - 1) / s_hat;
@@ -220,13 +231,22 @@ __device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_
   const int last_len = n_new - (nseg - 1) * s;
   const int kept_new = nseg > 0 ? (nseg - 1) * h + min(h, last_len) : 0;
   const int kept_mid = kept_old + kept_new;
+  const bool staged = evict_staged(pol);
 
   float* score = st.score + inst * pol.budget;
   int32_t* pos = st.pos + inst * pol.budget;
+  int32_t* src = work;
+  float* sc_s = reinterpret_cast<float*>(work + cap);
+  int32_t* pos_s = work + 2 * cap;
+  if (staged) {
+    for (int j = tid; j < m; j += THREADS) { sc_s[j] = score[mb + j]; pos_s[j] = pos[mb + j]; }
+    __syncthreads();
+  }
+  const float* sc = staged ? sc_s - mb : score;      // sc[slot] for slots of the middle region
 
   // ---- selection: src[t] = source slot of middle destination mb + t ---------------------------
   if (pol.policy == BUZZ_POLICY_GLOBAL_TOPK) {
-    topk_select<THREADS>(score + mb, n - mb, kept_mid, [&](int t, int j) { src[t] = mb + j; });
+    topk_select<THREADS>(sc + mb, m, kept_mid, [&](int t, int j) { src[t] = mb + j; });
   } else {
     for (int t = tid; t < kept_old; t += THREADS) src[t] = mb + t * s_hat;
     for (int seg = warp; seg < nseg; seg += THREADS / 32) {
@@ -243,7 +263,7 @@ __device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_
         Cand best{0.f, -1};
         for (int i = 0, j = lane; j < len; ++i, j += 32) {
           if (chosen >> i & 1u) continue;
-          best = better(best, Cand{score[lo + j], lo + j});
+          best = better(best, Cand{sc[lo + j], lo + j});
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
@@ -267,13 +287,21 @@ __device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_
   __syncthreads();
 
   // ---- compaction of score and pos ------------------------------------------------------------
-  for (int base = 0; base < kept_mid; base += THREADS) {
-    const int t = base + tid;
-    float sc = 0.f;
-    int32_t ps = 0;
-    if (t < kept_mid) { sc = score[src[t]]; ps = pos[src[t]]; }
-    __syncthreads();
-    if (t < kept_mid) { score[mb + t] = sc; pos[mb + t] = ps; }
+  if (staged) {                                      // sources are the shared-memory copies: no hazard
+    for (int t = tid; t < kept_mid; t += THREADS) {
+      const int j = src[t] - mb;
+      score[mb + t] = sc_s[j];
+      pos[mb + t] = pos_s[j];
+    }
+  } else {
+    for (int base = 0; base < kept_mid; base += THREADS) {
+      const int t = base + tid;
+      float v = 0.f;
+      int32_t ps = 0;
+      if (t < kept_mid) { v = score[src[t]]; ps = pos[src[t]]; }
+      __syncthreads();
+      if (t < kept_mid) { score[mb + t] = v; pos[mb + t] = ps; }
+    }
   }
 
   // ---- compaction of the K and V rows ---------------------------------------------------------

@@ -87,7 +87,7 @@ decode_kernel(BuzzState st, BuzzPolicy pol, const T* __restrict__ q, const T* __
   float* invL = fr + kMaxCluster * G;                        // [G]
   float* owarp = invL + G;                                   // [kWarps][G][D]
   float* sl = owarp + kWarps * G * D;                        // [G][chunk_cap]
-  int32_t* evict_src = reinterpret_cast<int32_t*>(sl + (size_t)G * chunk_cap);   // fused mode: [budget - sink - window]
+  int32_t* evict_src = reinterpret_cast<int32_t*>(sl + (size_t)G * chunk_cap);   // fused mode: work area of the eviction
 
   const int n0 = st.n[inst];
   const int tot = st.total[inst];
@@ -313,7 +313,7 @@ cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, con
   const int chunk_cap = (c->pol.budget + cluster_size - 1) / cluster_size;
   const size_t smem = sizeof(Partial<G, D>) +
                       sizeof(float) * (kWarps * G + kMaxCluster * G + G + kWarps * G * D + (size_t)G * chunk_cap) +
-                      (c->fused_evict ? sizeof(int32_t) * (size_t)(c->pol.budget - c->pol.sink - c->pol.window) : 0);
+                      (c->fused_evict ? buzz_dev::evict_smem_bytes(c->pol) : 0);
   static BuzzSmemOptIn opt_in;
   if (cudaError_t e = opt_in.ensure(decode_kernel<T, D, G>, smem); e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};

@@ -112,7 +112,7 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   float* invL = Mg + G;                                      // [G]
   float* owarp = invL + G;                                   // [kWarps][G][D]
   float* sl = owarp + kWarps * G * D;                        // [G][chunk_cap] logits (log2 domain)
-  int32_t* evict_src = reinterpret_cast<int32_t*>(sl + (size_t)G * chunk_cap);   // fused mode: [budget - sink - window]
+  int32_t* evict_src = reinterpret_cast<int32_t*>(sl + (size_t)G * chunk_cap);   // fused mode: work area of the eviction
 
   // Programmatic dependent launch; the host picks one of three modes.
   //   kWaitFirst  wait for everything earlier in the stream, then let the next launch begin.
@@ -428,7 +428,7 @@ cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, con
   const size_t smem = kStageBytes<D> + sizeof(Partial<G, D>) +
                       sizeof(float) * (kWarps * kHeads + kHeads + kMaxCluster * G + 2 * G +
                                        kWarps * G * D + (size_t)G * chunk_cap) +
-                      (c->fused_evict ? sizeof(int32_t) * (size_t)(c->pol.budget - c->pol.sink - c->pol.window) : 0);
+                      (c->fused_evict ? buzz_dev::evict_smem_bytes(c->pol) : 0);
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
   static BuzzSmemOptIn opt_in;
   if (cudaError_t e = opt_in.ensure(decode_bf16_kernel<D, G>, smem); e != cudaSuccess) return e;

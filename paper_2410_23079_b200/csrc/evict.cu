@@ -12,7 +12,7 @@ constexpr int kThreads = 256;
 template <int ROW_BYTES>
 __global__ void __launch_bounds__(kThreads)
 evict_kernel(BuzzState st, BuzzPolicy pol, int layer_begin, int max_batch, int kv_heads, int batch) {
-  extern __shared__ int32_t src[];   // source slot of every surviving middle slot
+  extern __shared__ int32_t src[];   // work area: source slot of every surviving middle slot, staged scores and positions
   const int head = blockIdx.x, seq = blockIdx.y, layer = layer_begin + blockIdx.z;
   if (seq >= batch) return;
   const size_t inst = ((size_t)layer * max_batch + seq) * kv_heads + head;
@@ -30,7 +30,7 @@ cudaError_t buzz_launch_evict(buzz_ctx* c, int layer_begin, int layer_count, cud
   if (batch == 0) return cudaSuccess;
   dim3 grid(c->sh.kv_heads, batch, layer_count);
   (void)cudaGetLastError();   // drop a stale non-sticky error left by an earlier runtime call of the process
-  const size_t smem = (size_t)(c->pol.budget - c->pol.sink - c->pol.window) * sizeof(int32_t);
+  const size_t smem = buzz_dev::evict_smem_bytes(c->pol);
   const int row_bytes = c->sh.head_dim * (int)c->esize;
 #define BUZZ_EVICT_CASE(RB)                                                                        \
   case RB: {                                                                                       \

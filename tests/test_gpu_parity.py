@@ -60,6 +60,34 @@ def test_logn_scaling(cuda_device):
     run_lockstep(w, [(0, 0, 0)], logn=True)
 
 
+@pytest.mark.parametrize("topk", [False, True])
+def test_eviction_with_a_middle_region_too_large_to_stage(cuda_device, topk):
+    """Middle regions beyond the size whose scores and positions the eviction copies to shared memory
+    take the path that selects straight from global memory; same bit-exact bar, both policies."""
+    rng = np.random.default_rng(77 + topk)
+    sink, window, segment, hitters, d = 4, 32, 16, 2, 64
+    T = 6000
+    budget = sink + window + T
+    w = workloads.scaled(workloads.get("C1"), batch=3, q_heads=1, kv_heads=1, sink=sink, window=window,
+                         segment=segment, hitters=hitters, budget=budget, head_dim=d, dtype="bf16")
+    bz = make_buzz(w, max_prompt_tokens=64)
+    bz.set_policy(topk)
+    cases = []
+    for b, n_old in enumerate([0, T // 2 + 3, T]):
+        pos, score, k, v = _random_state(rng, budget, d, torch.bfloat16, 7)
+        bz.import_state(0, b, 0, n_old, int(pos[-1]) + 1, torch.from_numpy(pos), torch.from_numpy(score), k, v)
+        orc = OracleHead(1, d, sink, window, segment, hitters, budget)
+        orc.set_policy(topk)
+        orc.set_state(n_old, int(pos[-1]) + 1, pos, score.astype(np.float64), k.double().numpy(), v.double().numpy())
+        cases.append((b, orc))
+    bz.evict(0)
+    assert bz.status() == 0
+    for b, orc in cases:
+        assert orc.evict() == 1
+        compare_state(bz, orc, 0, b, 0, f"large middle region b{b}", exact_scores=True)
+    bz.close()
+
+
 @pytest.mark.parametrize("name,over,samples", [
     ("C2", dict(layers=2, batch=2, q_heads=4, kv_heads=4, prompt_min=700, prompt_max=700, decode_steps=150,
                 window=64, budget=180), [(0, 0, 0), (1, 1, 3)]),
@@ -244,6 +272,34 @@ def test_eviction_bit_exact_on_planted_states(cuda_device, segment, hitters, qua
     bz.evict(-1)                       # a second call must be a no-op everywhere
     for b, h, orc, n in cases:
         compare_state(bz, orc, 0, b, h, f"planted again b{b} h{h}", exact_scores=True)
+    bz.close()
+
+
+@pytest.mark.parametrize("topk", [False, True])
+def test_eviction_with_a_middle_region_too_large_to_stage(cuda_device, topk):
+    """Middle regions beyond the size whose scores and positions the eviction copies to shared memory
+    take the path that selects straight from global memory; same bit-exact bar, both policies."""
+    rng = np.random.default_rng(77 + topk)
+    sink, window, segment, hitters, d = 4, 32, 16, 2, 64
+    T = 6000
+    budget = sink + window + T
+    w = workloads.scaled(workloads.get("C1"), batch=3, q_heads=1, kv_heads=1, sink=sink, window=window,
+                         segment=segment, hitters=hitters, budget=budget, head_dim=d, dtype="bf16")
+    bz = make_buzz(w, max_prompt_tokens=64)
+    bz.set_policy(topk)
+    cases = []
+    for b, n_old in enumerate([0, T // 2 + 3, T]):
+        pos, score, k, v = _random_state(rng, budget, d, torch.bfloat16, 7)
+        bz.import_state(0, b, 0, n_old, int(pos[-1]) + 1, torch.from_numpy(pos), torch.from_numpy(score), k, v)
+        orc = OracleHead(1, d, sink, window, segment, hitters, budget)
+        orc.set_policy(topk)
+        orc.set_state(n_old, int(pos[-1]) + 1, pos, score.astype(np.float64), k.double().numpy(), v.double().numpy())
+        cases.append((b, orc))
+    bz.evict(0)
+    assert bz.status() == 0
+    for b, orc in cases:
+        assert orc.evict() == 1
+        compare_state(bz, orc, 0, b, 0, f"large middle region b{b}", exact_scores=True)
     bz.close()
 
 
