@@ -138,6 +138,12 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");         // counters, q, k_new, v_new are read after this
   }
+  if (mode == kWaitFirst && rank == 0) {
+    // CTA 0's chunk starts at slot 0 whatever the length: pull its first rows towards L2 while the
+    // counters are on their way (a line of an unoccupied slot is fetched for nothing, never used)
+    const char* kb = reinterpret_cast<const char*>(st.K) + inst * (size_t)pol.budget * (D * 2);
+    if (tid * 128 < min(pol.budget, 64) * D * 2) asm volatile("prefetch.global.L2 [%0];" ::"l"(kb + (size_t)tid * 128));
+  }
   const int n0 = st.n[inst];
   const int tot = st.total[inst];
   const int ring_head = st.ring[inst];
@@ -355,7 +361,9 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   }
 
   // ---- combine across the cluster -------------------------------------------------------
-  cluster.sync();
+  // (a cluster of one CTA needs only the CTA barrier: a cluster barrier with release/acquire
+  // semantics also waits for the CTA's outstanding stores, about a microsecond each time)
+  if (C == 1) __syncthreads(); else cluster.sync();
   if (mode == kOverlap) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (rank == 0) {                   // every CTA has read n0/tot/ring and all old rows before the barrier
     if (tid <= 2 * NCH) cp_async_wait();
@@ -388,18 +396,30 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
   bool has_pending = false;
   {
     float* score = st.score + inst * pol.budget;
-    for (int j = tid; j < cnt; j += kThreads) {
-      float add = 0.f;
+    constexpr int U = 4;                             // slots per thread and pass: their old scores are fetched together
+    for (int j0 = tid; j0 < cnt; j0 += U * kThreads) {
+      float old[U];
 #pragma unroll
-      for (int g = 0; g < G; ++g) add += exp2f(sl[g * chunk_cap + j] - Mg[g]) * invL[g];
-      const int slot = lo + j;
-      if (slot == n0) {
-        if (app.slot_moved >= 0) { pending_score = add; has_pending = true; }
-        else score[n0] = add;
-      } else if (slot == app.slot_new) {             // only with a full ring: slot_new < n0
-        score[n0] = score[slot] + add;
-      } else {
-        score[slot] += add;
+      for (int u = 0; u < U; ++u) {
+        const int j = j0 + u * kThreads;
+        old[u] = (j < cnt && lo + j != n0) ? score[lo + j] : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int j = j0 + u * kThreads;
+        if (j >= cnt) break;
+        float add = 0.f;
+#pragma unroll
+        for (int g = 0; g < G; ++g) add += exp2f(sl[g * chunk_cap + j] - Mg[g]) * invL[g];
+        const int slot = lo + j;
+        if (slot == n0) {
+          if (app.slot_moved >= 0) { pending_score = add; has_pending = true; }
+          else score[n0] = add;
+        } else if (slot == app.slot_new) {           // only with a full ring: slot_new < n0
+          score[n0] = old[u] + add;
+        } else {
+          score[slot] = old[u] + add;
+        }
       }
     }
   }
@@ -412,7 +432,12 @@ decode_bf16_kernel(BuzzState st, BuzzPolicy pol, const __nv_bfloat16* __restrict
       o[idx] = __float2bfloat16_rn(acc * invL[g]);
     }
   }
-  cluster.sync();                    // peers may still be reading this CTA's shared memory
+  // Peers may still be reading this CTA's shared memory, and the thread that moves the leaving
+  // token's score must have read it before the pending store below. Only the fused eviction reads
+  // what OTHER CTAs of the cluster wrote to global memory, so only it needs release/acquire.
+  if (C == 1) __syncthreads();
+  else if (fused_evict) cluster.sync();
+  else asm volatile("barrier.cluster.arrive.relaxed.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
   if (has_pending) st.score[inst * pol.budget + app.slot_new] = pending_score;
   // Fused eviction (Algorithm 1's trigger: the cache is full after this step). Every score, row and
   // counter of the instance was written before the barrier above, by this cluster.
