@@ -293,12 +293,12 @@ def measure(w, K, W, peaks, dev, dist, world, *, headline, e2e_steps=0, evict_le
         # the method's own work per evicting instance: the score scan plus every surviving middle row read and written
         return sum(4 * (n - w.sink - w.window) + 2 * m2 * per_slot for (_, n, _, m2) in fired) * w.kv_heads * w.layers
 
-    def run_leg(step_fn, fused, steps, evict_call):
+    def run_leg(step_fn, fused, steps, evict_call, name=None):
         """`steps` steps; returns (ms, slot_sum, launches, evictions)."""
         bz.set_fused_evict(fused)
         slot_sum, ev = 0, 0
         l0 = bz.launch_count()
-        with Leg(stream) as leg:
+        with Leg(stream, name) as leg:
             for _ in range(steps):
                 step_fn()
                 if evict_call:
@@ -327,7 +327,7 @@ def measure(w, K, W, peaks, dev, dist, world, *, headline, e2e_steps=0, evict_le
     sampler = ClockSampler(dev.index or 0)
     sampler.start()
     time.sleep(0.3)
-    ms, slot_sum, launches, ev = run_leg(step_layers, True, K, False)
+    ms, slot_sum, launches, ev = run_leg(step_layers, True, K, False, "headline")
     if dist:
         dist.barrier()
     res["clocks"] = sampler.stop()
