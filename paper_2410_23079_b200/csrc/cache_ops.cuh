@@ -218,7 +218,7 @@ __host__ __device__ inline size_t evict_smem_bytes(const BuzzPolicy& p) {
 template <int ROW_BYTES, int THREADS>
 __device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_t inst, int n, int n_old,
                                int32_t* work) {
-  constexpr int kRowsPerPass = 4;   // rows of K and of V each 16-byte lane moves per pass
+  constexpr int kRowsPerPass = 2;   // rows of K and of V each 16-byte lane holds per register set (two sets in flight)
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int s = pol.segment, h = pol.hitters, s_hat = pol.s_hat;
   const int mb = middle_begin(pol);
@@ -310,9 +310,11 @@ __device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_
   uint4* Kc = reinterpret_cast<uint4*>(st.K + inst * (size_t)pol.budget * ROW_BYTES);
   uint4* Vc = reinterpret_cast<uint4*>(st.V + inst * (size_t)pol.budget * ROW_BYTES);
   const int sub = tid % LPR, rgrp = tid / LPR;
-  // Under the sampling policy the first old survivor stays where it is.
-  for (int base = (kept_old > 0 && pol.policy != BUZZ_POLICY_GLOBAL_TOPK) ? 1 : 0; base < kept_mid; base += ROWS) {
-    uint4 kr[kRowsPerPass], vr[kRowsPerPass];
+  // Under the sampling policy the first old survivor stays where it is. The loop is software-pipelined
+  // over two register sets: a chunk's destinations lie in front of every later chunk's sources
+  // (destination mb + t <= mb + t' <= src[t'] for t < t'), so the NEXT chunk's loads may be issued before
+  // this chunk is written; only a chunk's own loads have to be done (the barrier) before its stores.
+  auto load_rows = [&](int base, uint4 (&kr)[kRowsPerPass], uint4 (&vr)[kRowsPerPass]) {
 #pragma unroll
     for (int u = 0; u < kRowsPerPass; ++u) {
       const int t = base + u * (THREADS / LPR) + rgrp;
@@ -322,7 +324,8 @@ __device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_
         vr[u] = Vc[(size_t)sj * LPR + sub];
       }
     }
-    __syncthreads();
+  };
+  auto store_rows = [&](int base, const uint4 (&kr)[kRowsPerPass], const uint4 (&vr)[kRowsPerPass]) {
 #pragma unroll
     for (int u = 0; u < kRowsPerPass; ++u) {
       const int t = base + u * (THREADS / LPR) + rgrp;
@@ -331,6 +334,20 @@ __device__ void evict_instance(const BuzzState& st, const BuzzPolicy& pol, size_
         Vc[(size_t)(mb + t) * LPR + sub] = vr[u];
       }
     }
+  };
+  uint4 ka[kRowsPerPass], va[kRowsPerPass], kb[kRowsPerPass], vb[kRowsPerPass];
+  int base = (kept_old > 0 && pol.policy != BUZZ_POLICY_GLOBAL_TOPK) ? 1 : 0;
+  load_rows(base, ka, va);
+  while (base < kept_mid) {                          // uniform over the CTA
+    load_rows(base + ROWS, kb, vb);
+    __syncthreads();
+    store_rows(base, ka, va);
+    base += ROWS;
+    if (base >= kept_mid) break;
+    load_rows(base + ROWS, ka, va);
+    __syncthreads();
+    store_rows(base, kb, vb);
+    base += ROWS;
   }
 
   if (tid == 0) {
