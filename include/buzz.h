@@ -167,7 +167,9 @@ int buzz_decode_step_host(buzz_t ctx, int layer, const void* q_host, const void*
  * that batches independent attention calls. `layers` (host array of `count` pairwise distinct
  * layer indices) is walked in order; q, k_new, v_new and out are host arrays of `count` device
  * pointers with the layouts of buzz_decode_step for each layer's own batch. Results are those of
- * `count` buzz_decode_step calls.
+ * `count` buzz_decode_step calls: bit for bit when the cluster size is fixed with
+ * buzz_set_decode_cluster; with the built-in choice the two entry points may split an instance's
+ * slots over a different number of CTAs, which changes the fp32 summation order and nothing else.
  * Contract: every input buffer must be complete (in stream order) before this call, and no `out`
  * buffer may alias another member's buffers. Within the call the launches are NOT serialised:
  * CTAs of consecutive layers occupy the SMs back to back and each member finishes only after the

@@ -603,6 +603,7 @@ def test_decode_layers_matches_single_layer_calls(cuda_device, shape):
     pre, dec = _stack(w)
     ref, multi, host, paged = make_buzz(w), make_buzz(w), make_buzz(w), make_buzz(w)
     for bz in (ref, multi, host, paged):
+        bz.set_decode_cluster(2)          # same split of the slots in both entry points: bit-identical sums
         for l in range(w.layers):
             q, k, v, cu = pre[l]
             bz.prefill(l, q, k, v, cu, 150, torch.empty_like(q))
@@ -753,6 +754,7 @@ def test_decode_layers_with_uneven_and_empty_layers(cuda_device):
     ref, multi = make_buzz(w), make_buzz(w)
     nb = {0: 3, 1: 0, 2: 2}                                    # sequences per layer (layer 1 stays empty)
     for bz in (ref, multi):
+        bz.set_decode_cluster(1)
         for l, b in nb.items():
             if b:
                 q, k, v, cu = pre[l]
