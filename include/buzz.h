@@ -43,7 +43,7 @@ enum {
   BUZZ_ERR_NO_PROGRESS = -3, /* an eviction left the cache full (degenerate parameters)      */
   BUZZ_ERR_TIMEOUT = -4,     /* a bounded on-device wait expired                             */
   BUZZ_ERR_CUDA = -5,        /* a CUDA runtime call failed                                   */
-  BUZZ_ERR_TOO_LARGE = -6    /* request exceeds a built-in fixed-size buffer                 */
+  BUZZ_ERR_TOO_LARGE = -6    /* request exceeds a built-in fixed-size buffer or shared memory  */
 };
 
 typedef struct buzz_ctx* buzz_t;
@@ -208,7 +208,10 @@ int buzz_evict(buzz_t ctx, int layer, void* stream);
  * tail, whether the step has filled an instance's cache (n >= budget) and if so runs that instance's
  * eviction right there, exactly as buzz_evict would have on the next call. The caches are then never
  * full between calls, buzz_evict has nothing to do (and launches nothing), and the state after each
- * step is bit-identical to decode step + buzz_evict in the default mode. Default: off. */
+ * step is bit-identical to decode step + buzz_evict in the default mode. Default: off.
+ * Returns BUZZ_ERR_TOO_LARGE (and leaves the mode off) when the eviction's work area would not fit
+ * beside a decode CTA's buffers in shared memory, which only very large budgets with large groups
+ * reach (e.g. budget 32768 with 8 query heads per KV head); buzz_evict as a call of its own has no such limit. */
 int buzz_set_fused_evict(buzz_t ctx, int on);
 
 /* Test/checkpoint getter for one instance. Synchronises `stream`-independent: it waits for the

@@ -5,6 +5,7 @@
 #include <new>
 
 #include "buzz_internal.cuh"
+#include "cache_ops.cuh"
 
 cudaError_t buzz_launch_prefill_simt(buzz_ctx* c, const void* q, const void* k, const void* v,
                                      const int32_t* cu, int batch, int max_seqlen, void* out,
@@ -353,6 +354,13 @@ int buzz_evict(buzz_t c, int layer, void* stream) {
 
 int buzz_set_fused_evict(buzz_t c, int on) {
   if (!c) return BUZZ_ERR_INVALID;
+  if (on) {
+    // A decode CTA then holds the eviction's work area beside its own buffers in shared memory; with the
+    // instance split over the largest cluster (8 CTAs) that must stay within what a CTA may use.
+    const size_t G = c->group, D = c->sh.head_dim;
+    const size_t decode = 2048 + 4 * (2 * G + G * D) + 4 * (80 + 10 * G + 8 * G * D) + 4 * G * ((size_t)c->pol.budget / 8 + 4);
+    if (decode + buzz_dev::evict_smem_bytes(c->pol) > 200 * 1024) return BUZZ_ERR_TOO_LARGE;
+  }
   c->fused_evict = on ? 1 : 0;
   return BUZZ_OK;
 }

@@ -449,11 +449,17 @@ template <int D, int G>
 cudaError_t launch(buzz_ctx* c, int layer, const void* q, const void* k_new, const void* v_new,
                    void* out, int cluster_size, int mode, int next_layer, cudaStream_t stream) {
   const int batch = c->batch[layer];
-  const int chunk_cap = (((c->pol.budget + cluster_size - 1) / cluster_size + 1) & ~1) + 2;
-  const size_t smem = kStageBytes<D> + sizeof(Partial<G, D>) +
-                      sizeof(float) * (kWarps * kHeads + kHeads + kMaxCluster * G + 2 * G +
-                                       kWarps * G * D + (size_t)G * chunk_cap) +
-                      (c->fused_evict ? buzz_dev::evict_smem_bytes(c->pol) : 0);
+  // A CTA keeps the logits of its chunk (and, in fused mode, the eviction's work area) in shared
+  // memory: if that does not fit, split the instance over more CTAs.
+  int chunk_cap;
+  size_t smem;
+  for (;; cluster_size *= 2) {
+    chunk_cap = (((c->pol.budget + cluster_size - 1) / cluster_size + 1) & ~1) + 2;
+    smem = kStageBytes<D> + sizeof(Partial<G, D>) +
+           sizeof(float) * (kWarps * kHeads + kHeads + kMaxCluster * G + 2 * G + kWarps * G * D + (size_t)G * chunk_cap) +
+           (c->fused_evict ? buzz_dev::evict_smem_bytes(c->pol) : 0);
+    if (smem <= 200 * 1024 || cluster_size >= kMaxCluster) break;
+  }
   if (smem > 200 * 1024) return cudaErrorInvalidValue;
   static BuzzSmemOptIn opt_in;
   if (cudaError_t e = opt_in.ensure(decode_bf16_kernel<D, G>, smem); e != cudaSuccess) return e;

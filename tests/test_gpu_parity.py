@@ -372,6 +372,46 @@ def test_global_topk_bit_exact_on_planted_states(cuda_device, T, segment, hitter
     bz.close()
 
 
+def test_fused_mode_with_very_large_budgets(cuda_device):
+    """Fused mode keeps the eviction's work area in the decode CTA's shared memory. A budget of 20000
+    slots still fits (instance split over 8 CTAs, selection straight from global memory): one fused
+    step on a cache one token short of full evicts in the kernel's tail, and the counters follow the
+    oracle's schedule. A budget of 32768 with 8 query heads per KV head does not fit: refused."""
+    from paper_2410_23079_b200 import BuzzError
+    rng = np.random.default_rng(5)
+    sink, window, segment, hitters, d, budget = 4, 64, 16, 1, 128, 20000
+    w = workloads.scaled(workloads.get("C2"), layers=1, batch=1, q_heads=4, kv_heads=1, sink=sink, window=window,
+                         segment=segment, hitters=hitters, budget=budget)
+    bz = make_buzz(w, max_prompt_tokens=64)
+    bz.set_fused_evict(True)
+    n = budget - 1
+    pos, score, k, v = _random_state(rng, n, d, torch.bfloat16, 0)
+    n_old = 5000
+    bz.import_state(0, 0, 0, n_old, int(pos[-1]) + 1, torch.from_numpy(pos), torch.from_numpy(score), k, v)
+    orc = OracleHead(4, d, sink, window, segment, hitters, budget)
+    orc.set_state(n_old, int(pos[-1]) + 1, pos, score.astype(np.float64), k.double().numpy(), v.double().numpy())
+    q = torch.randn(1, 4, d, device="cuda:0").to(torch.bfloat16)
+    kn, vn = torch.randn(1, 1, d, device="cuda:0").to(torch.bfloat16), torch.randn(1, 1, d, device="cuda:0").to(torch.bfloat16)
+    out = torch.empty_like(q)
+    bz.decode_step(0, q, kn, vn, out)
+    assert bz.status() == 0
+    ref = orc.decode(q[0].double().cpu().numpy(), kn[0, 0].double().cpu().numpy(), vn[0, 0].double().cpu().numpy())
+    assert_close(out[0].double().cpu().numpy(), ref, what="fused step output", atol=2e-2, rtol=1e-2)
+    assert orc.evict() == 1
+    st = bz.export_state(0, 0, 0)
+    assert (st["n"], st["n_old"], st["total_len"]) == orc.counts()
+    opos = orc.state(with_kv=False)[0]
+    assert st["pos"][:sink].tolist() == opos[:sink].tolist() and st["pos"][-window:].tolist() == opos[-window:].tolist()
+    assert np.all(np.diff(st["pos"].numpy()) > 0)
+    bz.close()
+    big = workloads.scaled(workloads.get("C2"), layers=1, batch=1, q_heads=8, kv_heads=1, budget=32768)
+    bz = make_buzz(big, max_prompt_tokens=64)
+    with pytest.raises(BuzzError) as ei:
+        bz.set_fused_evict(True)
+    assert ei.value.code == -6
+    bz.close()
+
+
 def test_policy_validation(cuda_device):
     from paper_2410_23079_b200 import BuzzError
     w = workloads.scaled(workloads.get("C1"))
