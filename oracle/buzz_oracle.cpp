@@ -31,7 +31,7 @@
 //                                far: row index + 1 at prefill, total length incl. the new token at
 //                                decode -- not the number of retained slots).
 //
-// Readings taken where the paper is silent or inconsistent (each also listed in the design notes):
+// Readings taken where the paper is silent or inconsistent:
 //   T is the capacity of the middle region, budget = T + k + w (Remark 2, Fig. 3 caption);
 //   eviction fires when n >= budget; argmax ties go to the lowest position; a partial last
 //   segment is a short segment; interval sampling keeps offsets 0, s_hat, 2 s_hat, ...;
